@@ -1,0 +1,168 @@
+/*
+ * tlq.h - C ABI of libtlq: the hot path of TLQ's layer-wise calibration on one B200 (sm_100a).
+ *
+ * For one linear layer Y = X W^T + b (X: N tokens x C1 input channels, W: C2 x C1), every candidate
+ * r_k = k/K of the ratio grid gives a per-input-channel scale = x_stat^r_k (paper Sec. 3.1.2, first
+ * equation; Sec. 3.2.1, first equation).  The scaled weights are fake-quantized (Sec. 2.2 quantizer),
+ * the quantized layer f_q = Q_w(W*scale) Q_a(x/scale) + b is applied to the calibration tokens and
+ * the squared output error against f_fp = W x + b (Sec. 3.2.1, objective) is reduced per token with
+ * the token-importance weights (Sec. 3.1: gradient-derived importance; a 0/1 weight vector is the
+ * paper's top-50% token selection, a constant vector its plain expectation).  The argmin is kept.
+ *
+ * Conventions
+ *  - Every pointer is a DEVICE pointer unless its comment says "host".  The caller owns all buffers;
+ *    the library allocates and frees no device memory.  bf16 tensors are raw uint16 bit patterns,
+ *    row-major, innermost dimension contiguous.  X, W and the workspace must be 16-byte aligned
+ *    (TMA base-address rule) and C1 must be a multiple of 8 (16-byte row pitch).
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls validate
+ *    their arguments on the host, enqueue kernels on `stream` and return without synchronising.
+ *  - Return value: TLQ_OK or a negative TLQ_ERR_* for errors found on the host.  Errors found on
+ *    the device (a bounded wait that ran out, a grid whose losses are all non-finite) are written
+ *    to the int32 status word at byte 0 of the workspace; tlq_read_status() synchronises the stream
+ *    and returns it.
+ *  - There is no CPU fallback: without a CUDA device every compute call returns TLQ_ERR_CUDA.
+ */
+#ifndef TLQ_H_
+#define TLQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define TLQ_OK 0
+#define TLQ_ERR_INVALID_ARG (-1) /* NULL pointer, bad enum, bad struct_size */
+#define TLQ_ERR_SHAPE (-2)       /* N<1, C1%8, C1%group, K outside [1,64], ... */
+#define TLQ_ERR_ALIGN (-3)       /* a pointer that must be 16-byte aligned is not */
+#define TLQ_ERR_UNSUPPORTED (-4) /* bit width / mode combination not built */
+#define TLQ_ERR_WORKSPACE (-5)   /* workspace_bytes smaller than tlq_*_workspace_bytes() */
+#define TLQ_ERR_CUDA (-6)        /* a CUDA runtime / driver call failed (no device, launch error) */
+#define TLQ_ERR_TIMEOUT (-7)     /* device: a bounded barrier wait expired; results are invalid */
+#define TLQ_ERR_NONFINITE (-8)   /* device: every candidate's loss was non-finite */
+
+/* tlq_config.mode */
+#define TLQ_W4A16_ASYM_GROUP 0 /* weights: w_bits (2..8) asymmetric, one step + integer zero-point per
+                                  `group_size` consecutive input channels of an output row; activations
+                                  stay bf16 (Q_a = identity) */
+#define TLQ_W8A8_SYM 1         /* weights: int8 symmetric per output row; activations: int8 symmetric per
+                                  token, both with step max|.|/127 (Sec. 2.2, first two equations) */
+
+/* tlq_config.stat_mode: x_stat over the calibration tokens */
+#define TLQ_STAT_MEAN_ABS 0   /* mean_n |X_nc| (x_mean row of the paper's ablation table) */
+#define TLQ_STAT_MAX_ABS 1    /* max_n |X_nc| (x_max row) */
+#define TLQ_STAT_MASKED_MAX 2 /* max over the selected tokens I (Sec. 3.1.2, second equation) */
+
+/* tlq_token_importance: norm_kind, g_dtype */
+#define TLQ_NORM_MEAN_ABS 0 /* mean over channels of |g| (the text of Sec. 3.1.2) */
+#define TLQ_NORM_L2 1       /* ||g||_2 (the equation of Sec. 3.1.2 read as a Euclidean norm) */
+#define TLQ_DTYPE_BF16 0
+#define TLQ_DTYPE_F32 1
+
+#define TLQ_MAX_GRID 64
+
+typedef struct {
+  uint32_t struct_size; /* sizeof(tlq_config); checked */
+  int32_t mode;         /* TLQ_W4A16_ASYM_GROUP | TLQ_W8A8_SYM */
+  int32_t w_bits;       /* 2..8 for the group mode (codes are one per byte), 8 for W8A8 */
+  int32_t a_bits;       /* 16 for the group mode, 8 for W8A8 */
+  int32_t group_size;   /* 32, 64, 128 or 256 for the group mode (must divide C1); ignored for W8A8 */
+  int32_t n_grid;       /* K >= 1; candidate k uses r_k = k / K, so candidate 0 is scale = 1 */
+  int32_t stat_mode;    /* TLQ_STAT_* */
+  uint32_t flags;       /* reserved, must be 0 */
+} tlq_config;
+
+/* Stages of tlq_scale_search_layer, for tlq_stage_timing_read(). */
+#define TLQ_STAGE_STATS 0     /* x_stat and the K x C1 scale table */
+#define TLQ_STAGE_FAKEQUANT 1 /* operands of all K candidates (delta weights, or int8 weights + activations) */
+#define TLQ_STAGE_GEMM 2      /* fused tensor-core GEMM + per-token weighted error epilogue */
+#define TLQ_STAGE_REDUCE 3    /* losses, argmin, s_best, optional per-token table */
+#define TLQ_N_STAGES 4
+
+const char* tlq_status_string(int status);
+
+/* Version of this ABI (major*1000 + minor). */
+int tlq_version(void);
+
+/*
+ * Token importance (Sec. 3.1.2, third equation and the Top-50% selection):
+ *   imp[n] = sum_{b<B} norm(G[b,n,:]),  norm = mean_c |g| (TLQ_NORM_MEAN_ABS) or sqrt(sum_c g^2).
+ * If mask_out != NULL and top_frac > 0: mask_out[n] = 1 for the max(1, floor(top_frac*N)) positions
+ * with the largest imp (equal values: lower index first), else 0.
+ *   G        [B,N,C] bf16 bits or fp32 (g_dtype), C a multiple of 8
+ *   imp_out  [N] fp32            mask_out [N] uint8 or NULL
+ * Uses no scratch memory.
+ */
+int tlq_token_importance(const void* G, int g_dtype, int64_t B, int64_t N, int64_t C, int norm_kind,
+                         float top_frac, float* imp_out, uint8_t* mask_out, void* stream);
+
+/*
+ * Scale candidates (Sec. 3.1.2 first two equations; Table 2 variants):
+ *   x_stat[c] per cfg->stat_mode (mask [N] uint8 is read only for TLQ_STAT_MASKED_MAX),
+ *   m = max(x_stat, 2^-20),  s[k,c] = bf16(m^(k/K)).
+ *   X [N,C1] bf16; x_stat_out [C1] fp64 or NULL; s_out [K,C1] bf16
+ *   workspace: at least tlq_scale_candidates_workspace_bytes(N, C1) bytes (partial sums).
+ */
+size_t tlq_scale_candidates_workspace_bytes(int64_t N, int64_t C1);
+int tlq_scale_candidates(const void* X, int64_t N, int64_t C1, const uint8_t* mask, const tlq_config* cfg,
+                         void* workspace, size_t workspace_bytes, double* x_stat_out, void* s_out,
+                         void* stream);
+
+/*
+ * Fake-quantize the scaled weights for ONE scale vector: Q_w(W * scale) (Sec. 3.2.1, f_q; quantizer Sec. 2.2).
+ *   W [C2,C1] bf16;  s [C1] bf16 or NULL (= all ones, plain round-to-nearest)
+ * Group mode: codes [C2,C1] uint8 in [0,2^w_bits-1]; steps [C2,C1/G] fp32; zeros [C2,C1/G] int32;
+ *             dW_out [C2,C1] bf16 or NULL: W - dequant/scale (the tensor-core operand of the search).
+ * W8A8 mode:  codes [C2,C1] int8 bits; steps [C2] fp32; zeros ignored (may be NULL); dW_out must be NULL.
+ * Any of codes/steps/zeros may be NULL when not wanted.
+ */
+int tlq_quantize_weights(const void* W, const void* s, int64_t C2, int64_t C1, const tlq_config* cfg,
+                         uint8_t* codes, float* steps, int32_t* zeros, void* dW_out, void* stream);
+
+/*
+ * The layer-wise search (Sec. 3.2.1): for k in [0,K): loss[k] = sum_n w_n e_{k,n} / (C2 * sum_n w_n),
+ * e_{k,n} = || f_fp(x_n) - f_q(x_n; scale_k) ||_2^2; best_idx = argmin (lowest index on ties).
+ *   X [N,C1] bf16, W [C2,C1] bf16, w_imp [N] fp32 >= 0 or NULL (uniform),
+ *   mask [N] uint8 or NULL (token selection for TLQ_STAT_MASKED_MAX only),
+ *   best_idx [1] int32, losses [K] fp64, s_best [C1] bf16 (the winning scale),
+ *   per_token_err [K,N] fp32 or NULL (e_{k,n}).
+ * The workspace holds the operands of all K candidates; its status word is reset by this call.
+ */
+size_t tlq_scale_search_workspace_bytes(int64_t N, int64_t C1, int64_t C2, const tlq_config* cfg);
+int tlq_scale_search_layer(const void* X, int64_t N, int64_t C1, const void* W, int64_t C2,
+                           const float* w_imp, const uint8_t* mask, const tlq_config* cfg, void* workspace,
+                           size_t workspace_bytes, int32_t* best_idx, double* losses, void* s_best,
+                           float* per_token_err, void* stream);
+
+/*
+ * Apply the quantized layer with a chosen scale: Y_q = f_q(X; s) (+ bias), the activation the next
+ * layer calibrates on under the paper's adopted propagation strategy (Sec. 3.2.1, PassAct2).
+ *   s [C1] bf16 or NULL; bias [C2] bf16 or NULL; Yq [N,C2] bf16 (C2 a multiple of 8);
+ *   codes/steps/zeros as in tlq_quantize_weights (NULL = not wanted).
+ */
+size_t tlq_apply_layer_workspace_bytes(int64_t N, int64_t C1, int64_t C2, const tlq_config* cfg);
+int tlq_apply_layer(const void* X, int64_t N, int64_t C1, const void* W, int64_t C2, const void* s,
+                    const void* bias, const tlq_config* cfg, void* workspace, size_t workspace_bytes,
+                    uint8_t* codes, float* steps, int32_t* zeros, void* Yq, void* stream);
+
+/* Synchronise `stream` and return the device status word of `workspace` (TLQ_OK, TLQ_ERR_TIMEOUT,
+ * TLQ_ERR_NONFINITE) or TLQ_ERR_CUDA if the stream reports an error. */
+int tlq_read_status(const void* workspace, void* stream);
+
+/*
+ * Per-stage device timing of tlq_scale_search_layer, for benchmarks.  When enabled, the call records
+ * CUDA events on its stream between stages (events are created on first use and kept).  _read()
+ * synchronises on the last recorded event and writes TLQ_N_STAGES durations in milliseconds to the
+ * HOST array ms_out.  Off by default; not thread-safe.
+ */
+int tlq_stage_timing_enable(int on);
+int tlq_stage_timing_read(float* ms_out /* host [TLQ_N_STAGES] */);
+
+/* Number of kernels launched by this library since load (host counter; benchmarks report it). */
+int64_t tlq_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TLQ_H_ */

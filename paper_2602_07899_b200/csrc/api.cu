@@ -1,0 +1,319 @@
+// C ABI of libtlq: argument validation, workspace carving and stage sequencing.  All arithmetic of
+// the hot path lives in the kernels; nothing here computes on the host.
+#include <math.h>
+#include <string.h>
+
+#include "common.cuh"
+
+namespace tlq {
+
+long long g_launch_count = 0;
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_cfg(const tlq_config* cfg, int64_t C1, bool need_quantizer = true) {
+  if (cfg == nullptr || cfg->struct_size != sizeof(tlq_config)) return TLQ_ERR_INVALID_ARG;
+  if (cfg->flags != 0) return TLQ_ERR_INVALID_ARG;
+  if (cfg->n_grid < 1 || cfg->n_grid > TLQ_MAX_GRID) return TLQ_ERR_SHAPE;
+  if (cfg->stat_mode < TLQ_STAT_MEAN_ABS || cfg->stat_mode > TLQ_STAT_MASKED_MAX) return TLQ_ERR_INVALID_ARG;
+  if (C1 < 8 || (C1 % 8) != 0) return TLQ_ERR_SHAPE;
+  if (!need_quantizer) return TLQ_OK;
+  if (cfg->mode == TLQ_W4A16_ASYM_GROUP) {
+    if (cfg->w_bits < 2 || cfg->w_bits > 8 || cfg->a_bits != 16) return TLQ_ERR_UNSUPPORTED;
+    const int g = cfg->group_size;
+    if (g != 32 && g != 64 && g != 128 && g != 256) return TLQ_ERR_UNSUPPORTED;
+    if ((C1 % g) != 0) return TLQ_ERR_SHAPE;
+  } else if (cfg->mode == TLQ_W8A8_SYM) {
+    if (cfg->w_bits != 8 || cfg->a_bits != 8) return TLQ_ERR_UNSUPPORTED;
+    if ((C1 % 16) != 0 || C1 * 2 > 200 * 1024) return TLQ_ERR_SHAPE;
+  } else {
+    return TLQ_ERR_INVALID_ARG;
+  }
+  return TLQ_OK;
+}
+
+int have_device() {
+  int n = 0;
+  if (cudaGetDeviceCount(&n) != cudaSuccess || n < 1) {
+    cudaGetLastError();
+    return TLQ_ERR_CUDA;
+  }
+  return TLQ_OK;
+}
+
+// Carves consecutive 256-byte aligned regions out of a workspace (or only measures when base is null).
+struct Carver {
+  uint8_t* base;
+  size_t off;
+  explicit Carver(void* b) : base(reinterpret_cast<uint8_t*>(b)), off(0) {}
+  template <typename T>
+  T* take(size_t count, size_t align = 256) {
+    off = align_up(off, align);
+    T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off += count * sizeof(T);
+    return p;
+  }
+};
+
+struct SearchLayout {
+  WorkspaceHeader* hdr;
+  double* stat_partials;
+  double* x_stat;
+  uint16_t* s;
+  float* rs;
+  float* partials;
+  float* ptab;
+  uint16_t* dW;
+  int8_t* Wq;
+  float* u;
+  int8_t* Xq;
+  float* t;
+  size_t bytes;
+  GemmPlan plan;
+};
+
+SearchLayout carve_search(void* ws, int64_t N, int64_t C1, int64_t C2, const tlq_config* cfg) {
+  SearchLayout L{};
+  const int K = cfg->n_grid;
+  Carver c(ws);
+  L.plan = plan_search_gemm(N, C1, C2, K);
+  L.hdr = c.take<WorkspaceHeader>(1);
+  L.stat_partials = c.take<double>((size_t)stats_row_chunks(N) * C1);
+  L.x_stat = c.take<double>((size_t)C1);
+  L.s = c.take<uint16_t>((size_t)K * C1);
+  L.rs = c.take<float>((size_t)K * C1);
+  L.partials = c.take<float>((size_t)K * L.plan.partials_per_k);
+  L.ptab = c.take<float>((size_t)K * L.plan.otiles * L.plan.n_pad);
+  if (cfg->mode == TLQ_W4A16_ASYM_GROUP) {
+    L.dW = c.take<uint16_t>((size_t)K * C2 * C1, 1024);
+  } else {
+    L.Wq = c.take<int8_t>((size_t)K * C2 * C1, 1024);
+    L.u = c.take<float>((size_t)K * C2);
+    L.Xq = c.take<int8_t>((size_t)K * N * C1, 1024);
+    L.t = c.take<float>((size_t)K * N);
+  }
+  L.bytes = align_up(c.off, 256);
+  return L;
+}
+
+// ---------------------------------------------------------------------------------------------- stage timing
+bool g_timing_on = false;
+cudaEvent_t g_ev[TLQ_N_STAGES + 1] = {};
+bool g_ev_made = false;
+bool g_ev_valid = false;
+
+int timing_mark(int i, cudaStream_t st) {
+  if (!g_timing_on) return TLQ_OK;
+  if (!g_ev_made) {
+    for (int j = 0; j <= TLQ_N_STAGES; ++j) TLQ_CUDA_TRY(cudaEventCreate(&g_ev[j]));
+    g_ev_made = true;
+  }
+  TLQ_CUDA_TRY(cudaEventRecord(g_ev[i], st));
+  if (i == TLQ_N_STAGES) g_ev_valid = true;
+  return TLQ_OK;
+}
+
+}  // namespace
+}  // namespace tlq
+
+using namespace tlq;
+
+extern "C" {
+
+const char* tlq_status_string(int status) {
+  switch (status) {
+    case TLQ_OK: return "ok";
+    case TLQ_ERR_INVALID_ARG: return "invalid argument";
+    case TLQ_ERR_SHAPE: return "unsupported shape";
+    case TLQ_ERR_ALIGN: return "pointer not 16-byte aligned";
+    case TLQ_ERR_UNSUPPORTED: return "unsupported mode or bit width";
+    case TLQ_ERR_WORKSPACE: return "workspace too small";
+    case TLQ_ERR_CUDA: return "CUDA error or no CUDA device";
+    case TLQ_ERR_TIMEOUT: return "device-side wait timed out";
+    case TLQ_ERR_NONFINITE: return "all candidate losses are non-finite";
+    default: return "unknown status";
+  }
+}
+
+int tlq_version(void) { return 1000; }
+
+int64_t tlq_kernel_launch_count(void) { return (int64_t)g_launch_count; }
+
+int tlq_token_importance(const void* G, int g_dtype, int64_t B, int64_t N, int64_t C, int norm_kind, float top_frac,
+                         float* imp_out, uint8_t* mask_out, void* stream) {
+  if (G == nullptr || imp_out == nullptr) return TLQ_ERR_INVALID_ARG;
+  if (g_dtype != TLQ_DTYPE_BF16 && g_dtype != TLQ_DTYPE_F32) return TLQ_ERR_INVALID_ARG;
+  if (norm_kind != TLQ_NORM_MEAN_ABS && norm_kind != TLQ_NORM_L2) return TLQ_ERR_INVALID_ARG;
+  if (B < 1 || N < 1 || C < 8 || (C % 8) != 0 || N > 0x7FFFFFFFLL) return TLQ_ERR_SHAPE;
+  if (!(top_frac >= 0.0f) || top_frac > 1.0f) return TLQ_ERR_INVALID_ARG;
+  if (!aligned16(G)) return TLQ_ERR_ALIGN;
+  int rc = have_device();
+  if (rc != TLQ_OK) return rc;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  rc = launch_token_importance(G, g_dtype, B, N, C, norm_kind, imp_out, st);
+  if (rc != TLQ_OK) return rc;
+  if (mask_out != nullptr && top_frac > 0.0f) {
+    int64_t k_sel = (int64_t)floor((double)top_frac * (double)N);
+    if (k_sel < 1) k_sel = 1;
+    rc = launch_top_mask(imp_out, N, k_sel, mask_out, st);
+  }
+  return rc;
+}
+
+size_t tlq_scale_candidates_workspace_bytes(int64_t N, int64_t C1) {
+  if (N < 1 || C1 < 1) return 0;
+  return align_up((size_t)stats_row_chunks(N) * (size_t)C1 * sizeof(double), 256);
+}
+
+int tlq_scale_candidates(const void* X, int64_t N, int64_t C1, const uint8_t* mask, const tlq_config* cfg,
+                         void* workspace, size_t workspace_bytes, double* x_stat_out, void* s_out, void* stream) {
+  if (X == nullptr || workspace == nullptr || s_out == nullptr) return TLQ_ERR_INVALID_ARG;
+  if (N < 1) return TLQ_ERR_SHAPE;
+  int rc = check_cfg(cfg, C1, false);   // only the grid and the statistic are used here
+  if (rc != TLQ_OK) return rc;
+  if (cfg->stat_mode == TLQ_STAT_MASKED_MAX && mask == nullptr) return TLQ_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(workspace) || !aligned16(s_out)) return TLQ_ERR_ALIGN;
+  if (workspace_bytes < tlq_scale_candidates_workspace_bytes(N, C1)) return TLQ_ERR_WORKSPACE;
+  rc = have_device();
+  if (rc != TLQ_OK) return rc;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  double* partials = reinterpret_cast<double*>(workspace);
+  rc = launch_channel_stats(reinterpret_cast<const uint16_t*>(X), N, C1, mask, cfg->stat_mode, partials, st);
+  if (rc != TLQ_OK) return rc;
+  return launch_scale_table(partials, stats_row_chunks(N), N, C1, cfg->stat_mode, cfg->n_grid, x_stat_out,
+                            reinterpret_cast<uint16_t*>(s_out), nullptr, st);
+}
+
+int tlq_quantize_weights(const void* W, const void* s, int64_t C2, int64_t C1, const tlq_config* cfg, uint8_t* codes,
+                         float* steps, int32_t* zeros, void* dW_out, void* stream) {
+  if (W == nullptr) return TLQ_ERR_INVALID_ARG;
+  if (C2 < 1) return TLQ_ERR_SHAPE;
+  int rc = check_cfg(cfg, C1);
+  if (rc != TLQ_OK) return rc;
+  if (!aligned16(W) || (s != nullptr && !aligned16(s)) || (codes != nullptr && !aligned16(codes)) ||
+      (dW_out != nullptr && !aligned16(dW_out)))
+    return TLQ_ERR_ALIGN;
+  rc = have_device();
+  if (rc != TLQ_OK) return rc;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const uint16_t* Wb = reinterpret_cast<const uint16_t*>(W);
+  const uint16_t* sb = reinterpret_cast<const uint16_t*>(s);
+  if (cfg->mode == TLQ_W4A16_ASYM_GROUP)
+    return launch_fakequant_group(Wb, sb, 1, C2, C1, cfg->group_size, cfg->w_bits, reinterpret_cast<uint16_t*>(dW_out),
+                                  codes, steps, zeros, st);
+  if (dW_out != nullptr || codes == nullptr || steps == nullptr) return TLQ_ERR_INVALID_ARG;
+  return launch_fakequant_rows_i8(Wb, sb, 1, C2, C1, reinterpret_cast<int8_t*>(codes), steps, st);
+}
+
+size_t tlq_scale_search_workspace_bytes(int64_t N, int64_t C1, int64_t C2, const tlq_config* cfg) {
+  if (N < 1 || C2 < 1 || check_cfg(cfg, C1) != TLQ_OK) return 0;
+  return carve_search(nullptr, N, C1, C2, cfg).bytes;
+}
+
+int tlq_scale_search_layer(const void* X, int64_t N, int64_t C1, const void* W, int64_t C2, const float* w_imp,
+                           const uint8_t* mask, const tlq_config* cfg, void* workspace, size_t workspace_bytes,
+                           int32_t* best_idx, double* losses, void* s_best, float* per_token_err, void* stream) {
+  if (X == nullptr || W == nullptr || workspace == nullptr || best_idx == nullptr || losses == nullptr)
+    return TLQ_ERR_INVALID_ARG;
+  if (N < 1 || C2 < 1 || N > 0x7FFFFF00LL || C2 > 0x7FFFFF00LL) return TLQ_ERR_SHAPE;
+  int rc = check_cfg(cfg, C1);
+  if (rc != TLQ_OK) return rc;
+  if (cfg->stat_mode == TLQ_STAT_MASKED_MAX && mask == nullptr) return TLQ_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(W) || !aligned16(workspace)) return TLQ_ERR_ALIGN;
+  if (cfg->mode == TLQ_W8A8_SYM) return TLQ_ERR_UNSUPPORTED;
+  SearchLayout L = carve_search(workspace, N, C1, C2, cfg);
+  if (workspace_bytes < L.bytes) return TLQ_ERR_WORKSPACE;
+  rc = have_device();
+  if (rc != TLQ_OK) return rc;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const uint16_t* Xb = reinterpret_cast<const uint16_t*>(X);
+  const uint16_t* Wb = reinterpret_cast<const uint16_t*>(W);
+  const int K = cfg->n_grid;
+
+  TLQ_CUDA_TRY(cudaMemsetAsync(L.hdr, 0, sizeof(WorkspaceHeader), st));
+  if ((rc = timing_mark(0, st)) != TLQ_OK) return rc;
+  if ((rc = launch_channel_stats(Xb, N, C1, mask, cfg->stat_mode, L.stat_partials, st)) != TLQ_OK) return rc;
+  if ((rc = launch_scale_table(L.stat_partials, stats_row_chunks(N), N, C1, cfg->stat_mode, K, L.x_stat, L.s, L.rs,
+                               st)) != TLQ_OK)
+    return rc;
+  if ((rc = timing_mark(1, st)) != TLQ_OK) return rc;
+  if ((rc = launch_fakequant_group(Wb, L.s, K, C2, C1, cfg->group_size, cfg->w_bits, L.dW, nullptr, nullptr, nullptr,
+                                   st)) != TLQ_OK)
+    return rc;
+  if ((rc = timing_mark(2, st)) != TLQ_OK) return rc;
+  float* ptab = (per_token_err != nullptr) ? L.ptab : nullptr;
+  if ((rc = launch_search_gemm_bf16(Xb, L.dW, w_imp, L.plan, L.partials, ptab, L.hdr, st)) != TLQ_OK) return rc;
+  if ((rc = timing_mark(3, st)) != TLQ_OK) return rc;
+  if ((rc = launch_loss_reduce(L.partials, L.plan.partials_per_k, K, w_imp, N, C2, L.s, C1, L.hdr, losses, best_idx,
+                               reinterpret_cast<uint16_t*>(s_best), st)) != TLQ_OK)
+    return rc;
+  if (per_token_err != nullptr)
+    if ((rc = launch_per_token_reduce(L.ptab, K, L.plan.otiles, L.plan.n_pad, N, per_token_err, st)) != TLQ_OK)
+      return rc;
+  return timing_mark(4, st);
+}
+
+size_t tlq_apply_layer_workspace_bytes(int64_t N, int64_t C1, int64_t C2, const tlq_config* cfg) {
+  if (N < 1 || C2 < 1 || check_cfg(cfg, C1) != TLQ_OK) return 0;
+  Carver c(nullptr);
+  c.take<WorkspaceHeader>(1);
+  c.take<uint16_t>((size_t)C2 * C1, 1024);
+  return align_up(c.off, 256);
+}
+
+int tlq_apply_layer(const void* X, int64_t N, int64_t C1, const void* W, int64_t C2, const void* s, const void* bias,
+                    const tlq_config* cfg, void* workspace, size_t workspace_bytes, uint8_t* codes, float* steps,
+                    int32_t* zeros, void* Yq, void* stream) {
+  if (X == nullptr || W == nullptr || workspace == nullptr || Yq == nullptr) return TLQ_ERR_INVALID_ARG;
+  if (N < 1 || C2 < 8 || (C2 % 8) != 0 || N > 0x7FFFFF00LL) return TLQ_ERR_SHAPE;
+  int rc = check_cfg(cfg, C1);
+  if (rc != TLQ_OK) return rc;
+  if (!aligned16(X) || !aligned16(W) || !aligned16(workspace) || !aligned16(Yq) || (s != nullptr && !aligned16(s)) ||
+      (codes != nullptr && !aligned16(codes)))
+    return TLQ_ERR_ALIGN;
+  if (cfg->mode == TLQ_W8A8_SYM) return TLQ_ERR_UNSUPPORTED;
+  if (workspace_bytes < tlq_apply_layer_workspace_bytes(N, C1, C2, cfg)) return TLQ_ERR_WORKSPACE;
+  rc = have_device();
+  if (rc != TLQ_OK) return rc;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  Carver c(workspace);
+  WorkspaceHeader* hdr = c.take<WorkspaceHeader>(1);
+  uint16_t* dW = c.take<uint16_t>((size_t)C2 * C1, 1024);
+  const uint16_t* Xb = reinterpret_cast<const uint16_t*>(X);
+  const uint16_t* Wb = reinterpret_cast<const uint16_t*>(W);
+  TLQ_CUDA_TRY(cudaMemsetAsync(hdr, 0, sizeof(WorkspaceHeader), st));
+  if ((rc = launch_fakequant_group(Wb, reinterpret_cast<const uint16_t*>(s), 1, C2, C1, cfg->group_size, cfg->w_bits,
+                                   dW, codes, steps, zeros, st)) != TLQ_OK)
+    return rc;
+  return launch_apply_gemm_bf16(Xb, Wb, dW, reinterpret_cast<const uint16_t*>(bias), N, C1, C2,
+                                reinterpret_cast<uint16_t*>(Yq), hdr, st);
+}
+
+int tlq_read_status(const void* workspace, void* stream) {
+  if (workspace == nullptr) return TLQ_ERR_INVALID_ARG;
+  if (have_device() != TLQ_OK) return TLQ_ERR_CUDA;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (cudaStreamSynchronize(st) != cudaSuccess) return TLQ_ERR_CUDA;
+  int32_t status = 0;
+  if (cudaMemcpy(&status, workspace, sizeof(status), cudaMemcpyDeviceToHost) != cudaSuccess) return TLQ_ERR_CUDA;
+  return status;
+}
+
+int tlq_stage_timing_enable(int on) {
+  g_timing_on = on != 0;
+  g_ev_valid = false;
+  return TLQ_OK;
+}
+
+int tlq_stage_timing_read(float* ms_out) {
+  if (ms_out == nullptr) return TLQ_ERR_INVALID_ARG;
+  if (!g_timing_on || !g_ev_valid) return TLQ_ERR_INVALID_ARG;
+  if (cudaEventSynchronize(g_ev[TLQ_N_STAGES]) != cudaSuccess) return TLQ_ERR_CUDA;
+  for (int i = 0; i < TLQ_N_STAGES; ++i)
+    if (cudaEventElapsedTime(&ms_out[i], g_ev[i], g_ev[i + 1]) != cudaSuccess) return TLQ_ERR_CUDA;
+  return TLQ_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,122 @@
+// Shared declarations of the libtlq kernels (device helpers, launch bookkeeping, stage launchers).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "tlq.h"
+
+namespace tlq {
+
+// ---------------------------------------------------------------------------------------------
+// Host-side bookkeeping
+// ---------------------------------------------------------------------------------------------
+extern long long g_launch_count;  // kernels launched since load
+
+#define TLQ_CUDA_TRY(expr)                         \
+  do {                                             \
+    cudaError_t e__ = (expr);                      \
+    if (e__ != cudaSuccess) return TLQ_ERR_CUDA;   \
+  } while (0)
+
+inline int after_launch() {
+  ++g_launch_count;
+  return cudaGetLastError() == cudaSuccess ? TLQ_OK : TLQ_ERR_CUDA;
+}
+
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Floors on degenerate statistics (a dead channel, a flat group, a zero row).
+constexpr double kStatFloor = 9.5367431640625e-07;  // 2^-20
+#define TLQ_RANGE_FLOOR 1e-5f
+
+// ---------------------------------------------------------------------------------------------
+// Device helpers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t bits16) { return __uint_as_float(bits16 << 16); }
+
+// float -> bf16 bits, round to nearest even (finite inputs).
+__device__ __forceinline__ uint32_t float_to_bf16_bits(float f) {
+  uint32_t u = __float_as_uint(f);
+  u += 0x7FFFu + ((u >> 16) & 1u);
+  return u >> 16;
+}
+
+// Unpack 8 bf16 values held in a uint4 (little-endian pairs).
+__device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
+  f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xFFFF0000u);
+  f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xFFFF0000u);
+  f[4] = __uint_as_float(v.z << 16); f[5] = __uint_as_float(v.z & 0xFFFF0000u);
+  f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xFFFF0000u);
+}
+
+__device__ __forceinline__ uint4 ld_nc_16(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Workspace header (first 256 bytes of every workspace)
+// ---------------------------------------------------------------------------------------------
+struct WorkspaceHeader {
+  int32_t status;     // TLQ_OK / TLQ_ERR_TIMEOUT / TLQ_ERR_NONFINITE
+  int32_t where;      // diagnostic: which wait gave up
+  int32_t best_idx;   // device copy of the argmin
+  int32_t pad[61];
+};
+static_assert(sizeof(WorkspaceHeader) == 256, "header is 256 bytes");
+
+// ---------------------------------------------------------------------------------------------
+// Stage launchers (each enqueues on `st`, returns TLQ_OK or TLQ_ERR_CUDA)
+// ---------------------------------------------------------------------------------------------
+
+// stats.cu
+int64_t stats_row_chunks(int64_t N);
+int launch_channel_stats(const uint16_t* X, int64_t N, int64_t C1, const uint8_t* mask, int stat_mode,
+                         double* partials /*[chunks,C1]*/, cudaStream_t st);
+int launch_scale_table(const double* partials, int64_t chunks, int64_t N, int64_t C1, int stat_mode, int K,
+                       double* x_stat /*[C1] or null*/, uint16_t* s /*[K,C1]*/, float* rs /*[K,C1] or null*/,
+                       cudaStream_t st);
+
+// fakequant.cu
+int launch_fakequant_group(const uint16_t* W, const uint16_t* s /*[K,C1] or null*/, int K, int64_t C2, int64_t C1,
+                           int group, int w_bits, uint16_t* dW /*[K,C2,C1] or null*/, uint8_t* codes, float* steps,
+                           int32_t* zeros, cudaStream_t st);
+int launch_fakequant_rows_i8(const uint16_t* W, const uint16_t* s /*[K,C1] or null*/, int K, int64_t C2, int64_t C1,
+                             int8_t* q /*[K,C2,C1]*/, float* u /*[K,C2]*/, cudaStream_t st);
+int launch_actquant_i8(const uint16_t* X, const float* rs /*[K,C1] or null*/, int K, int64_t N, int64_t C1,
+                       int8_t* q /*[K,N,C1]*/, float* t /*[K,N]*/, cudaStream_t st);
+
+// importance.cu
+int launch_token_importance(const void* G, int g_dtype, int64_t B, int64_t N, int64_t C, int norm_kind,
+                            float* imp, cudaStream_t st);
+int launch_top_mask(const float* imp, int64_t N, int64_t k_sel, uint8_t* mask, cudaStream_t st);
+
+// reduce.cu
+int launch_loss_reduce(const float* partials, int64_t per_k, int K, const float* w_imp, int64_t N, int64_t C2,
+                       const uint16_t* s_table, int64_t C1, WorkspaceHeader* hdr, double* losses, int32_t* best_idx,
+                       uint16_t* s_best, cudaStream_t st);
+int launch_per_token_reduce(const float* ptab /*[K,otiles,Npad]*/, int K, int64_t otiles, int64_t Npad, int64_t N,
+                            float* per_token /*[K,N]*/, cudaStream_t st);
+
+// search_gemm.cu
+struct GemmPlan {
+  int64_t N, C1, C2;
+  int K;
+  int64_t mtiles, otiles;   // tiles along tokens / output channels
+  int64_t partials_per_k;   // floats per candidate in the partial buffer
+  int64_t n_pad;            // mtiles * 128
+};
+GemmPlan plan_search_gemm(int64_t N, int64_t C1, int64_t C2, int K);
+// W4A16 search: partials[K][mtiles*otiles*4] (+ ptab[K][otiles][n_pad] if non-null)
+int launch_search_gemm_bf16(const uint16_t* X, const uint16_t* dW, const float* w_imp, const GemmPlan& plan,
+                            float* partials, float* ptab, WorkspaceHeader* hdr, cudaStream_t st);
+// Apply: Yq[N,C2] = X W^T - X dW^T (+bias), bf16 out
+int launch_apply_gemm_bf16(const uint16_t* X, const uint16_t* W, const uint16_t* dW, const uint16_t* bias,
+                           int64_t N, int64_t C1, int64_t C2, uint16_t* Yq, WorkspaceHeader* hdr, cudaStream_t st);
+
+}  // namespace tlq

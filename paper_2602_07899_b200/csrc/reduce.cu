@@ -1,0 +1,101 @@
+// Final reduction of the search: loss[k] = sum_n w_n e_{k,n} / (C2 * sum_n w_n) (the expectation in
+// the objective of paper Sec. 3.2.1 with per-token importance weights), argmin with the lowest index
+// on ties, and the copy of the winning scale row.  Latency-bound: one CTA, fp64, fixed summation
+// order (per-thread strided serial sums, then a binary tree in shared memory), so two runs give
+// bit-identical losses.
+#include "common.cuh"
+
+namespace tlq {
+
+constexpr int kRedThreads = 1024;
+
+__device__ __forceinline__ double block_sum_fixed(double v, double* scratch) {
+  const int t = threadIdx.x;
+  __syncthreads();
+  scratch[t] = v;
+  __syncthreads();
+  for (int half = kRedThreads / 2; half > 0; half >>= 1) {
+    if (t < half) scratch[t] += scratch[t + half];
+    __syncthreads();
+  }
+  return scratch[0];
+}
+
+__global__ void __launch_bounds__(kRedThreads)
+loss_reduce_kernel(const float* __restrict__ partials, int64_t per_k, int K, const float* __restrict__ w_imp,
+                   int64_t N, int64_t C2, const uint16_t* __restrict__ s_table, int64_t C1, WorkspaceHeader* hdr,
+                   double* __restrict__ losses, int32_t* __restrict__ best_idx, uint16_t* __restrict__ s_best) {
+  __shared__ double scratch[kRedThreads];
+  __shared__ double loss_sh[TLQ_MAX_GRID];
+  __shared__ int best_sh;
+  const int t = threadIdx.x;
+
+  double wsum;
+  if (w_imp != nullptr) {
+    double a = 0.0;
+    for (int64_t n = t; n < N; n += kRedThreads) a += (double)w_imp[n];
+    wsum = block_sum_fixed(a, scratch);
+  } else {
+    wsum = (double)N;
+  }
+  const double denom = (double)C2 * wsum;
+
+  for (int k = 0; k < K; ++k) {
+    const float* p = partials + (int64_t)k * per_k;
+    double a = 0.0;
+    for (int64_t i = t; i < per_k; i += kRedThreads) a += (double)p[i];
+    const double total = block_sum_fixed(a, scratch);
+    if (t == 0) {
+      double l = total / denom;
+      if (!isfinite(l)) l = __longlong_as_double(0x7FF0000000000000LL);
+      loss_sh[k] = l;
+      losses[k] = l;
+    }
+  }
+  __syncthreads();
+  if (t == 0) {
+    int best = -1;
+    double bv = __longlong_as_double(0x7FF0000000000000LL);
+    for (int k = 0; k < K; ++k)
+      if (loss_sh[k] < bv) { bv = loss_sh[k]; best = k; }
+    if (best < 0) {
+      if (hdr->status == TLQ_OK) hdr->status = TLQ_ERR_NONFINITE;
+      best = 0;
+    }
+    best_sh = best;
+    hdr->best_idx = best;
+    *best_idx = best;
+  }
+  __syncthreads();
+  if (s_best != nullptr) {
+    const uint16_t* row = s_table + (int64_t)best_sh * C1;
+    for (int64_t c = t; c < C1; c += kRedThreads) s_best[c] = row[c];
+  }
+}
+
+__global__ void per_token_reduce_kernel(const float* __restrict__ ptab, int K, int64_t otiles, int64_t n_pad,
+                                        int64_t N, float* __restrict__ per_token) {
+  const int64_t n = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int k = blockIdx.y;
+  if (n >= N) return;
+  double a = 0.0;
+  for (int64_t o = 0; o < otiles; ++o) a += (double)ptab[((int64_t)k * otiles + o) * n_pad + n];
+  per_token[(int64_t)k * N + n] = (float)a;
+}
+
+int launch_loss_reduce(const float* partials, int64_t per_k, int K, const float* w_imp, int64_t N, int64_t C2,
+                       const uint16_t* s_table, int64_t C1, WorkspaceHeader* hdr, double* losses, int32_t* best_idx,
+                       uint16_t* s_best, cudaStream_t st) {
+  loss_reduce_kernel<<<1, kRedThreads, 0, st>>>(partials, per_k, K, w_imp, N, C2, s_table, C1, hdr, losses, best_idx,
+                                               s_best);
+  return after_launch();
+}
+
+int launch_per_token_reduce(const float* ptab, int K, int64_t otiles, int64_t n_pad, int64_t N, float* per_token,
+                            cudaStream_t st) {
+  dim3 grid((unsigned)ceil_div(N, 256), (unsigned)K);
+  per_token_reduce_kernel<<<grid, 256, 0, st>>>(ptab, K, otiles, n_pad, N, per_token);
+  return after_launch();
+}
+
+}  // namespace tlq

@@ -1,0 +1,252 @@
+"""ctypes binding of libtlq.so: same names as the C ABI (include/tlq.h), argument marshalling only.
+
+Tensors are torch CUDA tensors used purely as device-memory handles (bf16 tensors may be passed as
+torch.bfloat16 or as int16/uint16 bit patterns); the stream is torch's current stream unless given.
+Every step of the path runs in the library's kernels.  Importing this module loads the library and
+raises if it has not been built: there is no fallback implementation.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libtlq.so")
+
+OK = 0
+ERR_INVALID_ARG, ERR_SHAPE, ERR_ALIGN, ERR_UNSUPPORTED = -1, -2, -3, -4
+ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_NONFINITE = -5, -6, -7, -8
+W4A16_ASYM_GROUP, W8A8_SYM = 0, 1
+STAT_MEAN_ABS, STAT_MAX_ABS, STAT_MASKED_MAX = 0, 1, 2
+NORM_MEAN_ABS, NORM_L2 = 0, 1
+DTYPE_BF16, DTYPE_F32 = 0, 1
+N_STAGES = 4
+STAGE_NAMES = ("stats", "fakequant", "gemm", "reduce")
+
+EXPORTS = (
+    "tlq_status_string", "tlq_version", "tlq_token_importance", "tlq_scale_candidates_workspace_bytes",
+    "tlq_scale_candidates", "tlq_quantize_weights", "tlq_scale_search_workspace_bytes", "tlq_scale_search_layer",
+    "tlq_apply_layer_workspace_bytes", "tlq_apply_layer", "tlq_read_status", "tlq_stage_timing_enable",
+    "tlq_stage_timing_read", "tlq_kernel_launch_count",
+)
+
+
+class TlqError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: {status_string(status)} ({status})")
+
+
+class Config(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_uint32), ("mode", ctypes.c_int32), ("w_bits", ctypes.c_int32),
+                ("a_bits", ctypes.c_int32), ("group_size", ctypes.c_int32), ("n_grid", ctypes.c_int32),
+                ("stat_mode", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+
+
+def config(mode: int = W4A16_ASYM_GROUP, w_bits: Optional[int] = None, a_bits: Optional[int] = None,
+           group_size: int = 128, n_grid: int = 20, stat_mode: int = STAT_MEAN_ABS) -> Config:
+    if w_bits is None:
+        w_bits = 4 if mode == W4A16_ASYM_GROUP else 8
+    if a_bits is None:
+        a_bits = 16 if mode == W4A16_ASYM_GROUP else 8
+    return Config(ctypes.sizeof(Config), mode, w_bits, a_bits, group_size, n_grid, stat_mode, 0)
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2602_07899_b200.build` "
+                          "(there is no fallback implementation)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i64, i32, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_size_t
+    cfgp = ctypes.POINTER(Config)
+    lib.tlq_status_string.restype = ctypes.c_char_p
+    lib.tlq_status_string.argtypes = [i32]
+    lib.tlq_version.restype = i32
+    lib.tlq_kernel_launch_count.restype = i64
+    lib.tlq_token_importance.argtypes = [vp, i32, i64, i64, i64, i32, ctypes.c_float, vp, vp, vp]
+    lib.tlq_scale_candidates_workspace_bytes.restype = sz
+    lib.tlq_scale_candidates_workspace_bytes.argtypes = [i64, i64]
+    lib.tlq_scale_candidates.argtypes = [vp, i64, i64, vp, cfgp, vp, sz, vp, vp, vp]
+    lib.tlq_quantize_weights.argtypes = [vp, vp, i64, i64, cfgp, vp, vp, vp, vp, vp]
+    lib.tlq_scale_search_workspace_bytes.restype = sz
+    lib.tlq_scale_search_workspace_bytes.argtypes = [i64, i64, i64, cfgp]
+    lib.tlq_scale_search_layer.argtypes = [vp, i64, i64, vp, i64, vp, vp, cfgp, vp, sz, vp, vp, vp, vp, vp]
+    lib.tlq_apply_layer_workspace_bytes.restype = sz
+    lib.tlq_apply_layer_workspace_bytes.argtypes = [i64, i64, i64, cfgp]
+    lib.tlq_apply_layer.argtypes = [vp, i64, i64, vp, i64, vp, vp, cfgp, vp, sz, vp, vp, vp, vp, vp]
+    lib.tlq_read_status.argtypes = [vp, vp]
+    lib.tlq_stage_timing_enable.argtypes = [i32]
+    lib.tlq_stage_timing_read.argtypes = [ctypes.POINTER(ctypes.c_float)]
+    for fn in ("tlq_token_importance", "tlq_scale_candidates", "tlq_quantize_weights", "tlq_scale_search_layer",
+               "tlq_apply_layer", "tlq_read_status", "tlq_stage_timing_enable", "tlq_stage_timing_read"):
+        getattr(lib, fn).restype = i32
+    return lib
+
+
+lib = _load()
+
+
+def status_string(status: int) -> str:
+    return lib.tlq_status_string(int(status)).decode()
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_contiguous():
+        raise ValueError("tensor must be contiguous")
+    return t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _check(status: int, what: str) -> None:
+    if status != OK:
+        raise TlqError(status, what)
+
+
+def tlq_token_importance(G: torch.Tensor, norm_kind: int = NORM_MEAN_ABS, top_frac: float = 0.0,
+                         imp_out: Optional[torch.Tensor] = None, mask_out: Optional[torch.Tensor] = None, stream=None):
+    """G [B,N,C] (bf16 / int16 bits / float32) -> (imp float32 [N], mask uint8 [N] or None)."""
+    if G.dim() == 2:
+        G = G.unsqueeze(0)
+    B, N, C = G.shape
+    dt = DTYPE_F32 if G.dtype == torch.float32 else DTYPE_BF16
+    if imp_out is None:
+        imp_out = torch.empty(N, dtype=torch.float32, device=G.device)
+    if mask_out is None and top_frac > 0:
+        mask_out = torch.empty(N, dtype=torch.uint8, device=G.device)
+    _check(lib.tlq_token_importance(_ptr(G), dt, B, N, C, norm_kind, float(top_frac), _ptr(imp_out), _ptr(mask_out),
+                                    _stream(stream)), "tlq_token_importance")
+    return imp_out, mask_out
+
+
+def tlq_scale_candidates(X: torch.Tensor, cfg: Config, mask: Optional[torch.Tensor] = None, stream=None):
+    """X [N,C1] bf16 -> (x_stat float64 [C1], s bf16 [K,C1])."""
+    N, C1 = X.shape
+    nbytes = lib.tlq_scale_candidates_workspace_bytes(N, C1)
+    ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=X.device)
+    x_stat = torch.empty(C1, dtype=torch.float64, device=X.device)
+    s = torch.empty((cfg.n_grid, C1), dtype=torch.bfloat16, device=X.device)
+    _check(lib.tlq_scale_candidates(_ptr(X), N, C1, _ptr(mask), ctypes.byref(cfg), _ptr(ws), nbytes, _ptr(x_stat),
+                                    _ptr(s), _stream(stream)), "tlq_scale_candidates")
+    return x_stat, s
+
+
+def tlq_quantize_weights(W: torch.Tensor, s: Optional[torch.Tensor], cfg: Config, want_dw: bool = False, stream=None):
+    """W [C2,C1] bf16, s [C1] bf16 or None -> dict(codes, steps, zeros, dW)."""
+    C2, C1 = W.shape
+    dev = W.device
+    if cfg.mode == W4A16_ASYM_GROUP:
+        ng = C1 // cfg.group_size
+        codes = torch.empty((C2, C1), dtype=torch.uint8, device=dev)
+        steps = torch.empty((C2, ng), dtype=torch.float32, device=dev)
+        zeros = torch.empty((C2, ng), dtype=torch.int32, device=dev)
+        dW = torch.empty((C2, C1), dtype=torch.bfloat16, device=dev) if want_dw else None
+    else:
+        codes = torch.empty((C2, C1), dtype=torch.int8, device=dev)
+        steps = torch.empty((C2,), dtype=torch.float32, device=dev)
+        zeros, dW = None, None
+    _check(lib.tlq_quantize_weights(_ptr(W), _ptr(s), C2, C1, ctypes.byref(cfg), _ptr(codes), _ptr(steps), _ptr(zeros),
+                                    _ptr(dW), _stream(stream)), "tlq_quantize_weights")
+    return dict(codes=codes, steps=steps, zeros=zeros, dW=dW)
+
+
+def tlq_scale_search_workspace_bytes(N: int, C1: int, C2: int, cfg: Config) -> int:
+    return int(lib.tlq_scale_search_workspace_bytes(N, C1, C2, ctypes.byref(cfg)))
+
+
+class SearchBuffers:
+    """Caller-owned device buffers of one tlq_scale_search_layer call (reusable across calls)."""
+
+    def __init__(self, N: int, C1: int, C2: int, cfg: Config, device, per_token: bool = False,
+                 workspace: Optional[torch.Tensor] = None):
+        self.nbytes = tlq_scale_search_workspace_bytes(N, C1, C2, cfg)
+        if self.nbytes == 0:
+            raise TlqError(ERR_SHAPE, "tlq_scale_search_workspace_bytes")
+        if workspace is None or workspace.numel() < self.nbytes:
+            workspace = torch.empty(self.nbytes, dtype=torch.uint8, device=device)
+        self.workspace = workspace
+        self.best_idx = torch.empty(1, dtype=torch.int32, device=device)
+        self.losses = torch.empty(cfg.n_grid, dtype=torch.float64, device=device)
+        self.s_best = torch.empty(C1, dtype=torch.bfloat16, device=device)
+        self.per_token = torch.empty((cfg.n_grid, N), dtype=torch.float32, device=device) if per_token else None
+
+
+def tlq_scale_search_layer(X: torch.Tensor, W: torch.Tensor, w_imp: Optional[torch.Tensor], cfg: Config,
+                           buffers: Optional[SearchBuffers] = None, mask: Optional[torch.Tensor] = None,
+                           per_token: bool = False, stream=None, check: bool = True) -> SearchBuffers:
+    """Enqueue the search; with check=True also synchronise and raise on a device-side error."""
+    N, C1 = X.shape
+    C2 = W.shape[0]
+    if buffers is None:
+        buffers = SearchBuffers(N, C1, C2, cfg, X.device, per_token)
+    st = _stream(stream)
+    _check(lib.tlq_scale_search_layer(_ptr(X), N, C1, _ptr(W), C2, _ptr(w_imp), _ptr(mask), ctypes.byref(cfg),
+                                      _ptr(buffers.workspace), buffers.nbytes, _ptr(buffers.best_idx),
+                                      _ptr(buffers.losses), _ptr(buffers.s_best), _ptr(buffers.per_token), st),
+           "tlq_scale_search_layer")
+    if check:
+        _check(lib.tlq_read_status(_ptr(buffers.workspace), st), "tlq_scale_search_layer (device)")
+    return buffers
+
+
+def tlq_apply_layer(X: torch.Tensor, W: torch.Tensor, s: Optional[torch.Tensor], bias: Optional[torch.Tensor],
+                    cfg: Config, want_codes: bool = True, stream=None, check: bool = True):
+    """-> dict(Yq bf16 [N,C2], codes, steps, zeros)."""
+    N, C1 = X.shape
+    C2 = W.shape[0]
+    dev = X.device
+    nbytes = int(lib.tlq_apply_layer_workspace_bytes(N, C1, C2, ctypes.byref(cfg)))
+    if nbytes == 0:
+        raise TlqError(ERR_SHAPE, "tlq_apply_layer_workspace_bytes")
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    Yq = torch.empty((N, C2), dtype=torch.bfloat16, device=dev)
+    codes = steps = zeros = None
+    if want_codes:
+        if cfg.mode == W4A16_ASYM_GROUP:
+            ng = C1 // cfg.group_size
+            codes = torch.empty((C2, C1), dtype=torch.uint8, device=dev)
+            steps = torch.empty((C2, ng), dtype=torch.float32, device=dev)
+            zeros = torch.empty((C2, ng), dtype=torch.int32, device=dev)
+        else:
+            codes = torch.empty((C2, C1), dtype=torch.int8, device=dev)
+            steps = torch.empty((C2,), dtype=torch.float32, device=dev)
+    st = _stream(stream)
+    _check(lib.tlq_apply_layer(_ptr(X), N, C1, _ptr(W), C2, _ptr(s), _ptr(bias), ctypes.byref(cfg), _ptr(ws), nbytes,
+                               _ptr(codes), _ptr(steps), _ptr(zeros), _ptr(Yq), st), "tlq_apply_layer")
+    if check:
+        _check(lib.tlq_read_status(_ptr(ws), st), "tlq_apply_layer (device)")
+    return dict(Yq=Yq, codes=codes, steps=steps, zeros=zeros)
+
+
+def tlq_read_status(workspace: torch.Tensor, stream=None) -> int:
+    return int(lib.tlq_read_status(_ptr(workspace), _stream(stream)))
+
+
+def tlq_stage_timing_enable(on: bool) -> None:
+    _check(lib.tlq_stage_timing_enable(1 if on else 0), "tlq_stage_timing_enable")
+
+
+def tlq_stage_timing_read():
+    arr = (ctypes.c_float * N_STAGES)()
+    _check(lib.tlq_stage_timing_read(arr), "tlq_stage_timing_read")
+    return [float(v) for v in arr]
+
+
+def tlq_kernel_launch_count() -> int:
+    return int(lib.tlq_kernel_launch_count())
+
+
+def bf16_from_bits(bits, device="cuda") -> torch.Tensor:
+    """numpy uint16 bit patterns -> torch.bfloat16 device tensor (no arithmetic)."""
+    import numpy as np
+    t = torch.from_numpy(np.ascontiguousarray(bits).view(np.int16))
+    return t.to(device).view(torch.bfloat16)

@@ -1,0 +1,106 @@
+"""CPU-side checks: the C ABI library builds, loads and exports every declared symbol; host-side
+argument validation answers with error codes (no compute call reaches a GPU here)."""
+import ctypes
+import os
+import re
+
+import pytest
+import torch
+
+import __graft_entry__ as entry
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def tlq():
+    entry.build()
+    from paper_2602_07899_b200 import tlq as mod
+    return mod
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "tlq.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(tlq_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(tlq):
+    names = declared_symbols()
+    assert len(names) >= 12 and "tlq_scale_search_layer" in names
+    for n in names:
+        assert hasattr(tlq.lib, n), n
+    assert sorted(tlq.EXPORTS) == names
+    assert tlq.lib.tlq_version() == 1000
+    assert tlq.status_string(0) == "ok" and "workspace" in tlq.status_string(tlq.ERR_WORKSPACE)
+
+
+def test_config_struct_layout(tlq):
+    c = tlq.config()
+    assert ctypes.sizeof(tlq.Config) == 32 and c.struct_size == 32
+    assert (c.mode, c.w_bits, c.a_bits, c.group_size, c.n_grid) == (0, 4, 16, 128, 20)
+    c8 = tlq.config(tlq.W8A8_SYM)
+    assert (c8.w_bits, c8.a_bits) == (8, 8)
+
+
+def test_workspace_queries_and_shape_validation(tlq):
+    c = tlq.config()
+    n = tlq.tlq_scale_search_workspace_bytes(8192, 3584, 18944, c)
+    dW = 20 * 18944 * 3584 * 2
+    assert dW < n < dW + 400 * 2 ** 20
+    assert tlq.tlq_scale_search_workspace_bytes(256, 512, 512, c) % 256 == 0
+    assert tlq.tlq_scale_search_workspace_bytes(256, 500, 512, c) == 0          # C1 % 8
+    assert tlq.tlq_scale_search_workspace_bytes(256, 576, 512, c) == 0          # C1 % group
+    assert tlq.tlq_scale_search_workspace_bytes(0, 512, 512, c) == 0
+    bad = tlq.config(n_grid=65)
+    assert tlq.tlq_scale_search_workspace_bytes(256, 512, 512, bad) == 0
+    assert tlq.lib.tlq_scale_candidates_workspace_bytes(8192, 3584) >= 128 * 3584 * 8
+
+
+@pytest.mark.skipif(torch.cuda.is_available(), reason="checks the no-device error path")
+def test_compute_calls_fail_loudly_without_a_device(tlq):
+    c = tlq.config()
+    buf = (ctypes.c_uint8 * 4096)()
+    addr = (ctypes.addressof(buf) + 255) // 256 * 256
+    rc = tlq.lib.tlq_quantize_weights(addr, None, 8, 128, ctypes.byref(c), addr, addr, addr, None, None)
+    assert rc == tlq.ERR_CUDA
+    rc = tlq.lib.tlq_token_importance(addr, 0, 1, 4, 8, 0, 0.0, addr, None, None)
+    assert rc == tlq.ERR_CUDA
+
+
+def test_host_validation_error_codes(tlq):
+    c = tlq.config()
+    buf = (ctypes.c_uint8 * 8192)()
+    a = (ctypes.addressof(buf) + 255) // 256 * 256
+    L = tlq.lib
+    assert L.tlq_quantize_weights(None, None, 8, 128, ctypes.byref(c), a, a, a, None, None) == tlq.ERR_INVALID_ARG
+    assert L.tlq_quantize_weights(a + 2, None, 8, 128, ctypes.byref(c), a, a, a, None, None) == tlq.ERR_ALIGN
+    assert L.tlq_quantize_weights(a, None, 8, 100, ctypes.byref(c), a, a, a, None, None) == tlq.ERR_SHAPE
+    c3 = tlq.config(group_size=48)
+    assert L.tlq_quantize_weights(a, None, 8, 96, ctypes.byref(c3), a, a, a, None, None) == tlq.ERR_UNSUPPORTED
+    c.struct_size = 8
+    assert L.tlq_quantize_weights(a, None, 8, 128, ctypes.byref(c), a, a, a, None, None) == tlq.ERR_INVALID_ARG
+    c = tlq.config()
+    assert L.tlq_scale_search_layer(a, 4, 128, a, 8, None, None, ctypes.byref(c), a, 16, a, a, a, None,
+                                    None) == tlq.ERR_WORKSPACE
+    assert L.tlq_scale_search_layer(a, 4, 128, a, 8, None, None, ctypes.byref(c), None, 1 << 30, a, a, a, None,
+                                    None) == tlq.ERR_INVALID_ARG
+    cm = tlq.config(stat_mode=tlq.STAT_MASKED_MAX)
+    assert L.tlq_scale_search_layer(a, 4, 128, a, 8, None, None, ctypes.byref(cm), a, 1 << 30, a, a, a, None,
+                                    None) == tlq.ERR_INVALID_ARG
+    assert L.tlq_token_importance(a, 7, 1, 4, 8, 0, 0.0, a, None, None) == tlq.ERR_INVALID_ARG
+    assert L.tlq_token_importance(a, 0, 1, 4, 12, 0, 0.0, a, None, None) == tlq.ERR_SHAPE
+    assert L.tlq_token_importance(a, 0, 1, 4, 8, 0, 1.5, a, None, None) == tlq.ERR_INVALID_ARG
+    assert L.tlq_read_status(None, None) == tlq.ERR_INVALID_ARG
+    arr = (ctypes.c_float * 4)()
+    assert L.tlq_stage_timing_read(arr) == tlq.ERR_INVALID_ARG      # timing never enabled
+
+
+def test_oracle_never_imports_the_cuda_path():
+    for fn in ("tlq_oracle.py", "brute.py"):
+        src = open(os.path.join(ROOT, "oracle", fn)).read()
+        assert "paper_2602_07899_b200" not in src and "ctypes" not in src and "torch" not in src
+    for fn in os.listdir(os.path.join(ROOT, "paper_2602_07899_b200")):
+        if fn.endswith(".py"):
+            text = open(os.path.join(ROOT, "paper_2602_07899_b200", fn)).read()
+            assert not re.search(r"^\s*(from|import)\s+oracle", text, flags=re.M), fn

@@ -1,0 +1,245 @@
+"""GPU parity: the CUDA path (through the C ABI binding) against the CPU oracle, element by element on
+the same seeded inputs.  Integer work (codes, zero-points, scale bits, argmin) must match bit for bit;
+weighted losses and per-token errors within 2e-3 relative."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import tlq_oracle as orc
+from paper_2602_07899_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+LOSS_RTOL = 2e-3   # the stated tolerance on weighted losses (and per-token errors)
+
+
+@pytest.fixture(scope="module")
+def tlq():
+    import __graft_entry__ as entry
+    entry.build()
+    from paper_2602_07899_b200 import tlq as mod
+    return mod
+
+
+def dev_bf16(tlq, bits):
+    return tlq.bf16_from_bits(bits)
+
+
+def bits_of(t: torch.Tensor) -> np.ndarray:
+    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+# ----------------------------------------------------------------------------------- (a) statistics + scale table
+
+
+@pytest.mark.parametrize("n,c1", [(256, 512), (300, 264), (1, 8), (4100, 1544), (8192, 3584)])
+@pytest.mark.parametrize("stat", [0, 1, 2])
+def test_scale_candidates_bit_exact(tlq, n, c1, stat):
+    if stat == 2 and n == 8192:
+        pytest.skip("covered by the smaller shapes")
+    xb = wl.activations(5, f"sc/{n}x{c1}", n, c1, (3 * n) // 4, "normal", min(4, c1))
+    mask_np = (np.random.default_rng(n + c1).random(n) < 0.5).astype(np.uint8)
+    mask_np[0] = 1
+    cfg = tlq.config(stat_mode=stat, n_grid=20)
+    mask = torch.from_numpy(mask_np).cuda() if stat == 2 else None
+    x_stat, s = tlq.tlq_scale_candidates(dev_bf16(tlq, xb), cfg, mask)
+    torch.cuda.synchronize()
+    ref_stat = orc.channel_stat(xb, stat, mask_np)
+    ref_s = orc.scale_table(ref_stat, 20)
+    np.testing.assert_allclose(x_stat.cpu().numpy(), ref_stat, rtol=1e-14, atol=0)
+    assert np.array_equal(bits_of(s), orc.f32_to_bf16_bits(ref_s))
+
+
+# ----------------------------------------------------------------------------------- (b) fake-quant
+
+
+@pytest.mark.parametrize("c2,c1,group,bits", [(512, 512, 128, 4), (37, 384, 64, 4), (130, 1024, 256, 3),
+                                              (16, 96, 32, 8), (1, 128, 128, 2), (1000, 3584, 128, 4)])
+def test_group_quantizer_bit_exact(tlq, c2, c1, group, bits):
+    xb = wl.activations(7, f"gq/x{c1}", 64, c1, 48, "normal", 4)
+    wb = wl.weights(7, f"gq/w{c2}x{c1}", c2, c1)
+    s_np = orc.scale_table(orc.channel_stat(xb), 20)[13]
+    cfg = tlq.config(w_bits=bits, group_size=group)
+    for s_vec in (None, s_np):
+        s_dev = None if s_vec is None else dev_bf16(tlq, orc.f32_to_bf16_bits(s_vec))
+        out = tlq.tlq_quantize_weights(dev_bf16(tlq, wb), s_dev, cfg, want_dw=True)
+        torch.cuda.synchronize()
+        codes, step, zero, w_hat = orc.quantize_weights_group_asym(wb, s_vec, group, bits)
+        assert np.array_equal(out["codes"].cpu().numpy(), codes)
+        assert np.array_equal(out["zeros"].cpu().numpy(), zero)
+        assert np.array_equal(out["steps"].cpu().numpy().view(np.uint32), step.view(np.uint32))
+        assert np.array_equal(bits_of(out["dW"]), orc.delta_weights_bf16(wb, w_hat))
+
+
+def test_degenerate_groups(tlq):
+    # flat group, zero group, all-positive group, huge and tiny magnitudes
+    w = np.zeros((4, 256), dtype=np.float32)
+    w[0, :128] = 0.25
+    w[1, :128] = np.linspace(0.5, 1.0, 128)
+    w[2, 128:] = -np.linspace(1e-3, 2e-3, 128)
+    w[3, :] = np.random.default_rng(0).standard_normal(256) * 1e4
+    wb = wl.f32_to_bf16_bits(w)
+    cfg = tlq.config()
+    out = tlq.tlq_quantize_weights(dev_bf16(tlq, wb), None, cfg, want_dw=True)
+    torch.cuda.synchronize()
+    codes, step, zero, w_hat = orc.quantize_weights_group_asym(wb, None, 128)
+    assert np.array_equal(out["codes"].cpu().numpy(), codes)
+    assert np.array_equal(out["zeros"].cpu().numpy(), zero)
+    assert np.array_equal(out["steps"].cpu().numpy(), step)
+    assert np.array_equal(bits_of(out["dW"]), orc.delta_weights_bf16(wb, w_hat))
+
+
+@pytest.mark.parametrize("c2,c1", [(64, 512), (33, 1040), (512, 3584)])
+def test_int8_row_quantizer_bit_exact(tlq, c2, c1):
+    xb = wl.activations(9, f"i8/x{c1}", 32, c1, 24, "normal", 4)
+    wb = wl.weights(9, f"i8/w{c2}x{c1}", c2, c1)
+    s_np = orc.scale_table(orc.channel_stat(xb), 20)[7]
+    cfg = tlq.config(tlq.W8A8_SYM)
+    for s_vec in (None, s_np):
+        s_dev = None if s_vec is None else dev_bf16(tlq, orc.f32_to_bf16_bits(s_vec))
+        out = tlq.tlq_quantize_weights(dev_bf16(tlq, wb), s_dev, cfg)
+        torch.cuda.synchronize()
+        qw, u = orc.quantize_weights_row_sym(wb, s_vec)
+        assert np.array_equal(out["codes"].cpu().numpy(), qw)
+        assert np.array_equal(out["steps"].cpu().numpy().view(np.uint32), u.view(np.uint32))
+
+
+# ----------------------------------------------------------------------------------- (d) token importance
+
+
+@pytest.mark.parametrize("b,n,c,norm", [(6, 100, 64, 0), (3, 257, 520, 1), (1, 50, 8, 0), (16, 1058, 512, 0)])
+def test_token_importance(tlq, b, n, c, norm):
+    gb = wl.token_gradients(3, f"g/{b}x{n}x{c}", b, n, c, (3 * n) // 4)
+    imp, mask = tlq.tlq_token_importance(dev_bf16(tlq, gb), norm, 0.5)
+    torch.cuda.synchronize()
+    ref_imp, ref_mask = orc.token_importance(gb, norm, 0.5)
+    got = imp.cpu().numpy().astype(np.float64)
+    np.testing.assert_allclose(got, ref_imp, rtol=1e-5, atol=1e-30)
+    m = mask.cpu().numpy()
+    k_sel = max(1, n // 2)
+    assert m.sum() == k_sel
+    # the mask is exactly the top-k (ties: lower index) of the values the kernel itself produced
+    assert np.array_equal(m, orc.top_mask(imp.cpu().numpy(), 0.5))
+    # and agrees with the oracle's selection except where two importances are within rounding of the cut
+    diff = np.flatnonzero(m != ref_mask)
+    if diff.size:
+        cut = np.sort(ref_imp)[::-1][k_sel - 1]
+        assert np.all(np.abs(ref_imp[diff] - cut) <= 1e-5 * cut)
+    # float32 gradients take the same path
+    gf = torch.from_numpy(wl.bf16_bits_to_f32(gb)).cuda()
+    imp32, _ = tlq.tlq_token_importance(gf, norm, 0.0)
+    np.testing.assert_allclose(imp32.cpu().numpy(), got, rtol=1e-6)
+
+
+# ----------------------------------------------------------------------------------- (c) the search
+
+
+def run_search(tlq, xb, wb, imp, group=128, n_grid=20, w_bits=4, stat=0, mask=None):
+    cfg = tlq.config(w_bits=w_bits, group_size=group, n_grid=n_grid, stat_mode=stat)
+    w_dev = None if imp is None else torch.from_numpy(np.asarray(imp, dtype=np.float32)).cuda()
+    m_dev = None if mask is None else torch.from_numpy(mask).cuda()
+    out = tlq.tlq_scale_search_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), w_dev, cfg, mask=m_dev, per_token=True)
+    return dict(best=int(out.best_idx.item()), losses=out.losses.cpu().numpy(), per_token=out.per_token.cpu().numpy(),
+                s_best=bits_of(out.s_best))
+
+
+def check_against_oracle(got, ref, n_grid):
+    np.testing.assert_allclose(got["per_token"], ref["per_token"], rtol=LOSS_RTOL, atol=1e-30)
+    np.testing.assert_allclose(got["losses"], ref["losses"], rtol=LOSS_RTOL)
+    order = np.sort(ref["losses"])
+    gap = (order[1] - order[0]) / order[0] if n_grid > 1 else 1.0
+    if gap > 1e-5:
+        assert got["best"] == ref["best"]
+    else:   # the oracle's own two best candidates are closer than the arithmetic can tell apart
+        assert ref["losses"][got["best"]] <= order[0] * (1 + 1e-5)
+    assert got["best"] == int(np.argmin(got["losses"]))
+    assert np.array_equal(got["s_best"], orc.f32_to_bf16_bits(ref["scales"][got["best"]]))
+
+
+def test_search_cfg0(tlq):
+    cfgw = wl.config("cfg0")
+    data = wl.LayerData(cfgw)
+    lin = cfgw.linear("q")
+    ref = orc.scale_search(data.x(lin), data.w(lin), data.imp(), "w4a16", 128, 20)
+    got = run_search(tlq, data.x(lin), data.w(lin), data.imp())
+    check_against_oracle(got, ref, 20)
+
+
+@pytest.mark.parametrize("n,c1,c2,group,n_grid", [(300, 192, 320, 64, 5), (128, 64, 256, 32, 3), (1, 128, 64, 128, 2),
+                                                  (515, 1088, 777, 64, 7), (257, 512, 256, 256, 1)])
+def test_search_ragged_shapes(tlq, n, c1, c2, group, n_grid):
+    xb, wb, imp = wl.small_case(17, n, c1, c2, n_outlier=2)
+    ref = orc.scale_search(xb, wb, imp, "w4a16", group, n_grid)
+    got = run_search(tlq, xb, wb, imp, group, n_grid)
+    check_against_oracle(got, ref, n_grid)
+
+
+def test_search_importance_special_cases(tlq):
+    xb, wb, imp = wl.small_case(23, 384, 256, 512)
+    ref = orc.scale_search(xb, wb, None, "w4a16", 128, 6)
+    uni = run_search(tlq, xb, wb, None, 128, 6)
+    check_against_oracle(uni, ref, 6)
+    const = run_search(tlq, xb, wb, np.full(384, 2.5, np.float32), 128, 6)
+    np.testing.assert_allclose(const["losses"], uni["losses"], rtol=1e-6)            # uniform importance = plain MSE
+    hot = np.zeros(384, np.float32)
+    hot[201] = 3.0
+    one = run_search(tlq, xb, wb, hot, 128, 6)
+    np.testing.assert_allclose(one["losses"], uni["per_token"][:, 201].astype(np.float64) / 512.0, rtol=1e-6)
+    np.testing.assert_allclose(one["losses"], ref["per_token"][:, 201] / 512.0, rtol=LOSS_RTOL)
+    sel = np.zeros(384, np.float32)
+    sel[100:292] = 1.0                                                                # a 0/1 token selection
+    sub = run_search(tlq, xb, wb, sel, 128, 6)
+    np.testing.assert_allclose(sub["losses"], ref["per_token"][:, 100:292].mean(axis=1) / 512.0, rtol=LOSS_RTOL)
+
+
+def test_search_masked_max_statistic(tlq):
+    xb, wb, imp = wl.small_case(29, 200, 256, 256)
+    mask = orc.top_mask(imp.astype(np.float64), 0.5)
+    ref = orc.scale_search(xb, wb, imp, "w4a16", 128, 8, orc.STAT_MASKED_MAX, mask)
+    got = run_search(tlq, xb, wb, imp, 128, 8, stat=2, mask=mask)
+    check_against_oracle(got, ref, 8)
+
+
+def test_search_is_deterministic(tlq):
+    xb, wb, imp = wl.small_case(31, 640, 512, 768)
+    a = run_search(tlq, xb, wb, imp)
+    b = run_search(tlq, xb, wb, imp)
+    assert np.array_equal(a["losses"].view(np.uint64), b["losses"].view(np.uint64))
+    assert np.array_equal(a["per_token"].view(np.uint32), b["per_token"].view(np.uint32))
+
+
+def test_apply_layer(tlq):
+    xb, wb, imp = wl.small_case(37, 300, 256, 328)
+    ref = orc.scale_search(xb, wb, imp, "w4a16", 128, 8)
+    s = ref["scales"][ref["best"]]
+    bias_bits = wl.f32_to_bf16_bits(np.linspace(-0.5, 0.5, 328).astype(np.float32))
+    yq_ref, (codes, step, zero) = orc.apply_layer(xb, wb, s, bias_bits, "w4a16", 128)
+    out = tlq.tlq_apply_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), dev_bf16(tlq, orc.f32_to_bf16_bits(s)),
+                              dev_bf16(tlq, bias_bits), tlq.config())
+    assert np.array_equal(out["codes"].cpu().numpy(), codes)
+    assert np.array_equal(out["zeros"].cpu().numpy(), zero)
+    yq = out["Yq"].float().cpu().numpy().astype(np.float64)
+    # bf16 output rounding (half an ulp = 2^-9 relative, doubled for slack) plus the bf16 rounding of the
+    # delta-weight operand, which perturbs a token's output by a fraction of that token's rms output error
+    rms_e = np.sqrt(ref["per_token"][ref["best"]] / 328.0)[:, None]
+    err = np.abs(yq - yq_ref)
+    assert np.all(err <= 2.0 ** -8 * np.abs(yq_ref) + 5e-3 * rms_e + 1e-6)
+    # without scale and bias
+    out0 = tlq.tlq_apply_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), None, None, tlq.config(), want_codes=False)
+    y0_ref, _ = orc.apply_layer(xb, wb, None, None, "w4a16", 128)
+    y0 = out0["Yq"].float().cpu().numpy().astype(np.float64)
+    rms0 = np.sqrt(ref["per_token"][0] / 328.0)[:, None]
+    assert np.all(np.abs(y0 - y0_ref) <= 2.0 ** -8 * np.abs(y0_ref) + 5e-3 * rms0 + 1e-6)
+
+
+def test_device_errors_are_reported_not_raised_as_faults(tlq):
+    # host-side refusals on a live device: nothing is launched, the context stays usable
+    import ctypes
+    x = torch.zeros((4, 128), dtype=torch.bfloat16, device="cuda")
+    c = tlq.config()
+    ws = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    rc = tlq.lib.tlq_scale_search_layer(x.data_ptr(), 4, 128, x.data_ptr(), 4, None, None, ctypes.byref(c),
+                                        ws.data_ptr(), 1024, ws.data_ptr(), ws.data_ptr(), ws.data_ptr(), None, None)
+    assert rc == tlq.ERR_WORKSPACE
+    torch.cuda.synchronize()
+    assert tlq.tlq_kernel_launch_count() >= 0
