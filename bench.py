@@ -1,0 +1,365 @@
+#!/usr/bin/env python
+"""Benchmark of the TLQ scale-search hot path on B200.
+
+One "step" = the whole hot path over one decoder layer's seven linears (q, k, v, o, gate, up, down):
+per linear, activation statistics -> K scale candidates -> fake-quant of all candidates -> fused
+tensor-core GEMM with the importance-weighted error epilogue -> losses + argmin.  The metric is
+scale-grid candidates per second (7 linears x K candidates per step) plus the fused GEMM's TFLOP/s.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg1] [--impl ours|reference]
+
+N > 1 (torchrun): every rank calibrates its own layer (own seed), no data-path collective: weak scaling.
+`--impl reference` times the CPU oracle on a bounded sample of the same workload (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "scale_grid_candidates_per_sec"
+UNIT = "candidates/s"
+SAMPLE_LINEAR = "k"
+SAMPLE_TOKENS = 2048
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(bf16_sustained=float(p.get("bf16_tflops_sustained", 1400.0)), bf16_burst=float(p["bf16_tflops"]),
+                    hbm=float(p["hbm_gbs"]), source="measured")
+    return dict(bf16_sustained=1400.0, bf16_burst=1590.0, hbm=6650.0, source="fallback")
+
+
+def layer_flops(cfgw):
+    return sum(cfgw.flops_per_candidate(l) for l in cfgw.linears()) * cfgw.n_grid
+
+
+# --------------------------------------------------------------------------------------------- CPU oracle legs
+
+
+def oracle_sample_seconds(cfgw, data):
+    """One pass of the oracle over the bounded sample: one projection, the first SAMPLE_TOKENS tokens,
+    all K candidates.  Returns (seconds, flops of the sample)."""
+    from oracle import tlq_oracle as orc
+    lin = cfgw.linear(SAMPLE_LINEAR)
+    n = min(SAMPLE_TOKENS, cfgw.n_tokens)
+    x, w, imp = data.x(lin)[:n], data.w(lin), data.imp()[:n]
+    t0 = time.perf_counter()
+    orc.scale_search(x, w, imp, cfgw.mode, cfgw.group, cfgw.n_grid)
+    dt = time.perf_counter() - t0
+    return dt, 2.0 * n * lin.c_in * lin.c_out * cfgw.n_grid
+
+
+def sample_description(cfgw):
+    lin = cfgw.linear(SAMPLE_LINEAR)
+    n = min(SAMPLE_TOKENS, cfgw.n_tokens)
+    return (f"{SAMPLE_LINEAR}-projection {lin.c_in}->{lin.c_out}, first {n} of {cfgw.n_tokens} tokens, all "
+            f"{cfgw.n_grid} candidates; scaled to the whole layer by 2*N*C1*C2*K (extrapolated)")
+
+
+def candidates_per_sec_from_sample(cfgw, seconds, flops):
+    n_cand = len(cfgw.linears()) * cfgw.n_grid
+    return n_cand * (flops / layer_flops(cfgw)) / seconds
+
+
+def run_reference(args, cfgw):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2602_07899_b200 import workloads as wl
+    data = wl.LayerData(cfgw)
+    for _ in range(args.warmup):
+        oracle_sample_seconds(cfgw, data)
+    times = []
+    for _ in range(args.steps):
+        dt, flops = oracle_sample_seconds(cfgw, data)
+        times.append(dt)
+    total = sum(times)
+    value = candidates_per_sec_from_sample(cfgw, total / len(times), flops)
+    cores = os.cpu_count()
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": workload_name(cfgw), "sample": sample_description(cfgw)},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": sample_description(cfgw)},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def workload_name(cfgw):
+    return (f"{cfgw.key}: decoder layer hidden={cfgw.hidden} inter={cfgw.inter} kv={cfgw.kv}, {cfgw.n_tokens} tokens, "
+            f"{cfgw.mode} group={cfgw.group}, K={cfgw.n_grid}, 7 linears per step")
+
+
+# --------------------------------------------------------------------------------------------- clocks
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1])); pw.append(float(parts[2]))
+            except ValueError:
+                continue
+            for nme, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nme)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "power_w_max": max(pw), "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------------------------- GPU arm
+
+
+def run_ours(args, cfgw):
+    import torch
+    import torch.distributed as dist
+    from paper_2602_07899_b200 import tlq, workloads as wl
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # every rank calibrates its own layer: same shapes, its own seed
+    import dataclasses
+    cfgr = dataclasses.replace(cfgw, seed=cfgw.seed + rank)
+    data = wl.LayerData(cfgr)
+    lins = [l for l in cfgr.linears() if args.linears is None or l.name in args.linears.split(",")]
+    mode = tlq.W4A16_ASYM_GROUP if cfgr.mode == "w4a16" else tlq.W8A8_SYM
+    cfg = tlq.config(mode=mode, group_size=cfgr.group, n_grid=cfgr.n_grid)
+
+    # host (pinned) copies for the end-to-end leg, device-resident copies for the kernel leg
+    host_x, host_w, dev_x, dev_w = {}, {}, {}, {}
+    for l in lins:
+        if l.x_name not in host_x:
+            host_x[l.x_name] = torch.from_numpy(data.x(l).view(np.int16)).pin_memory()
+            dev_x[l.x_name] = host_x[l.x_name].to(dev, non_blocking=True).view(torch.bfloat16)
+        host_w[l.name] = torch.from_numpy(data.w(l).view(np.int16)).pin_memory()
+        dev_w[l.name] = host_w[l.name].to(dev, non_blocking=True).view(torch.bfloat16)
+    host_imp = torch.from_numpy(data.imp()).pin_memory()
+    dev_imp = host_imp.to(dev, non_blocking=True)
+    ws_bytes = max(tlq.tlq_scale_search_workspace_bytes(cfgr.n_tokens, l.c_in, l.c_out, cfg) for l in lins)
+    workspace = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    bufs = {l.name: tlq.SearchBuffers(cfgr.n_tokens, l.c_in, l.c_out, cfg, dev, False, workspace) for l in lins}
+    torch.cuda.synchronize()
+
+    def step(xs, ws, imp):
+        for l in lins:
+            tlq.tlq_scale_search_layer(xs[l.x_name], ws[l.name], imp, cfg, bufs[l.name], check=False)
+
+    for _ in range(args.warmup):
+        step(dev_x, dev_w, dev_imp)
+    st = tlq.tlq_read_status(workspace)
+    if st != tlq.OK:
+        raise SystemExit(f"device status after warm-up: {tlq.status_string(st)}")
+
+    # ---- kernel leg: inputs resident in HBM
+    sampler = ClockSampler(local)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sampler.start()
+    tlq.tlq_stage_timing_enable(True)
+    launches0 = tlq.tlq_kernel_launch_count()
+    ev0.record()
+    for _ in range(args.steps):
+        step(dev_x, dev_w, dev_imp)
+    ev1.record()
+    barrier()
+    clocks = sampler.stop()
+    launches = tlq.tlq_kernel_launch_count() - launches0
+    stage_ms = tlq.tlq_stage_timing_drain(512)
+    tlq.tlq_stage_timing_enable(False)
+    ms_total = ev0.elapsed_time(ev1)
+    st = tlq.tlq_read_status(workspace)
+    if st != tlq.OK:
+        raise SystemExit(f"device status after the timed region: {tlq.status_string(st)}")
+    best = {l.name: int(bufs[l.name].best_idx.item()) for l in lins}
+
+    # ---- end-to-end leg: host buffers in, results out, every step
+    if args.profile:
+        print(json.dumps({"profile_run": True, "ms_per_step": ms_total / args.steps, "stage_ms": stage_ms[-len(lins):]}))
+        return
+    x_stage = {k: torch.empty_like(v, device=dev) for k, v in host_x.items()}
+    w_stage = {k: torch.empty_like(v, device=dev) for k, v in host_w.items()}
+    imp_stage = torch.empty_like(dev_imp)
+    out_host = {l.name: (torch.empty(1, dtype=torch.int32).pin_memory(),
+                         torch.empty(cfgr.n_grid, dtype=torch.float64).pin_memory()) for l in lins}
+    h2d = sum(v.numel() * 2 for v in host_x.values()) + sum(v.numel() * 2 for v in host_w.values()) + host_imp.numel() * 4
+    d2h = len(lins) * (4 + 8 * cfgr.n_grid)
+
+    def e2e_step():
+        for k, v in host_x.items():
+            x_stage[k].copy_(v, non_blocking=True)
+        for k, v in host_w.items():
+            w_stage[k].copy_(v, non_blocking=True)
+        imp_stage.copy_(host_imp, non_blocking=True)
+        xs = {k: v.view(torch.bfloat16) for k, v in x_stage.items()}
+        wsd = {k: v.view(torch.bfloat16) for k, v in w_stage.items()}
+        step(xs, wsd, imp_stage)
+        for l in lins:
+            out_host[l.name][0].copy_(bufs[l.name].best_idx, non_blocking=True)
+            out_host[l.name][1].copy_(bufs[l.name].losses, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    ms_e2e = e0.elapsed_time(e1)
+    assert all(int(out_host[l.name][0].item()) == best[l.name] for l in lins)
+
+    # ---- max over ranks
+    if world > 1:
+        t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total, ms_e2e = float(t[0]), float(t[1])
+
+    n_cand_step = len(lins) * cfgr.n_grid
+    value = world * n_cand_step * args.steps / (ms_total * 1e-3)
+    e2e_value = world * n_cand_step * args.steps / (ms_e2e * 1e-3)
+
+    # ---- roofline of the dominant kernel (the fused search GEMM), from the per-stage events of the timed region
+    peaks = measured_peaks()
+    per_linear = {}
+    gemm_ms_sum, gemm_flops_sum = 0.0, 0.0
+    stage_tot = [0.0] * tlq.N_STAGES
+    for i, rec in enumerate(stage_ms):
+        l = lins[i % len(lins)]
+        fl = cfgr.flops_per_candidate(l) * cfgr.n_grid
+        d = per_linear.setdefault(l.name, {"gemm_ms": [], "flops": fl, "stages_ms": [0.0] * tlq.N_STAGES})
+        d["gemm_ms"].append(rec[2])
+        for j in range(tlq.N_STAGES):
+            d["stages_ms"][j] += rec[j]
+            stage_tot[j] += rec[j]
+        gemm_ms_sum += rec[2]
+        gemm_flops_sum += fl
+    n_rec = max(1, len(stage_ms) // len(lins))
+    lin_report = {}
+    for name, d in per_linear.items():
+        g = statistics.mean(d["gemm_ms"])
+        lin_report[name] = {"gemm_ms": round(g, 4), "gemm_tflops": round(d["flops"] / (g * 1e-3) / 1e12, 1),
+                            "stages_ms": [round(v / n_rec, 4) for v in d["stages_ms"]],
+                            "candidates_per_s": round(cfgr.n_grid / (sum(d["stages_ms"]) / n_rec * 1e-3), 1),
+                            "best_idx": best[name]}
+    achieved = gemm_flops_sum / (gemm_ms_sum * 1e-3) / 1e12 if gemm_ms_sum > 0 else None
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "search_gemm_traffic.json")
+    if os.path.exists(tpath):
+        with open(tpath) as f:
+            traffic = json.load(f).get(cfgr.key)
+    roofline = {"kernel": "gemm_bf16_kernel<search>", "bound": "tensor", "achieved": achieved,
+                "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
+                "frac": (achieved / peaks["bf16_sustained"]) if achieved else None, "traffic": traffic,
+                "peak_source": f"{peaks['source']} (sustained cuBLAS bf16; burst {peaks['bf16_burst']})",
+                "frac_of_nominal_2250": (achieved / 2250.0) if achieved else None,
+                "launches_timed": len(stage_ms),
+                "stage_share": {n: round(v / max(sum(stage_tot), 1e-9), 4) for n, v in zip(tlq.STAGE_NAMES, stage_tot)}}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    cpu = None
+    if world == 1:
+        dt, fl = oracle_sample_seconds(cfgw, data)
+        cpu = {"value": candidates_per_sec_from_sample(cfgw, dt, fl), "unit": UNIT, "cores": os.cpu_count(),
+               "kind": "oracle", "sample": sample_description(cfgw), "sample_seconds": round(dt, 3),
+               "oracle_gflops": round(fl / dt / 1e9, 1)}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if cfgr.mode == "w4a16" else "int8", "data": "synthetic",
+            "config": {"workload": workload_name(cfgr) + ("" if args.linears is None else f" [subset: {args.linears}]"), "l2": "inputs_exceed_l2 (operands of one linear: 0.1-2.9 GB)",
+                       "parallelism": f"replicas x{world} (one layer per rank, no collective)"},
+            "gemm_tflops": achieved, "roofline": roofline, "cpu_baseline": cpu,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": ms_e2e / args.steps},
+            "gpu_launches": launches, "clocks": clocks, "per_linear": lin_report}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="cfg1")
+    ap.add_argument("--linears", default=None, help="comma-separated subset of q,k,v,o,gate,up,down (profiling)")
+    ap.add_argument("--profile", action="store_true", help="kernel leg only: skip the end-to-end and CPU legs")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    from paper_2602_07899_b200 import workloads as wl
+    cfgw = wl.config(args.config)
+    if args.impl == "reference":
+        run_reference(args, cfgw)
+    else:
+        run_ours(args, cfgw)
+
+
+if __name__ == "__main__":
+    main()

@@ -73,7 +73,7 @@ typedef struct {
   uint32_t flags;       /* reserved, must be 0 */
 } tlq_config;
 
-/* Stages of tlq_scale_search_layer, for tlq_stage_timing_read(). */
+/* Stages of tlq_scale_search_layer, for tlq_stage_timing_drain(). */
 #define TLQ_STAGE_STATS 0     /* x_stat and the K x C1 scale table */
 #define TLQ_STAGE_FAKEQUANT 1 /* operands of all K candidates (delta weights, or int8 weights + activations) */
 #define TLQ_STAGE_GEMM 2      /* fused tensor-core GEMM + per-token weighted error epilogue */
@@ -151,13 +151,15 @@ int tlq_apply_layer(const void* X, int64_t N, int64_t C1, const void* W, int64_t
 int tlq_read_status(const void* workspace, void* stream);
 
 /*
- * Per-stage device timing of tlq_scale_search_layer, for benchmarks.  When enabled, the call records
- * CUDA events on its stream between stages (events are created on first use and kept).  _read()
- * synchronises on the last recorded event and writes TLQ_N_STAGES durations in milliseconds to the
- * HOST array ms_out.  Off by default; not thread-safe.
+ * Per-stage device timing of tlq_scale_search_layer, for benchmarks.  While enabled, every search call
+ * records CUDA events on its stream between its stages (event sets come from a pool of 512 created on
+ * first use; further calls are not recorded).  _drain() synchronises on the recorded events, writes
+ * TLQ_N_STAGES durations in milliseconds per recorded call, oldest first, to the HOST array ms_out
+ * (room for max_calls calls), forgets them and returns how many calls it wrote (or a negative
+ * TLQ_ERR_*).  _enable() also forgets what was recorded.  Off by default; not thread-safe.
  */
 int tlq_stage_timing_enable(int on);
-int tlq_stage_timing_read(float* ms_out /* host [TLQ_N_STAGES] */);
+int tlq_stage_timing_drain(float* ms_out /* host [max_calls][TLQ_N_STAGES] */, int max_calls);
 
 /* Number of kernels launched by this library since load (host counter; benchmarks report it). */
 int64_t tlq_kernel_launch_count(void);

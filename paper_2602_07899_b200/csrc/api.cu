@@ -99,19 +99,28 @@ SearchLayout carve_search(void* ws, int64_t N, int64_t C1, int64_t C2, const tlq
 }
 
 // ---------------------------------------------------------------------------------------------- stage timing
+// A fixed pool of event sets, one per recorded call; calls beyond the pool are not recorded.
+constexpr int kMaxTimedCalls = 512;
 bool g_timing_on = false;
-cudaEvent_t g_ev[TLQ_N_STAGES + 1] = {};
-bool g_ev_made = false;
-bool g_ev_valid = false;
+cudaEvent_t (*g_ev)[TLQ_N_STAGES + 1] = nullptr;   // [kMaxTimedCalls][5], created on first use
+int g_ev_made = 0;      // sets whose events exist
+int g_calls = 0;        // calls recorded since the last enable
+int g_cur = -1;         // set being recorded by the call in progress
 
 int timing_mark(int i, cudaStream_t st) {
   if (!g_timing_on) return TLQ_OK;
-  if (!g_ev_made) {
-    for (int j = 0; j <= TLQ_N_STAGES; ++j) TLQ_CUDA_TRY(cudaEventCreate(&g_ev[j]));
-    g_ev_made = true;
+  if (i == 0) {
+    if (g_calls >= kMaxTimedCalls) { g_cur = -1; return TLQ_OK; }
+    if (g_ev == nullptr) g_ev = new cudaEvent_t[kMaxTimedCalls][TLQ_N_STAGES + 1];
+    if (g_calls >= g_ev_made) {
+      for (int j = 0; j <= TLQ_N_STAGES; ++j) TLQ_CUDA_TRY(cudaEventCreate(&g_ev[g_ev_made][j]));
+      ++g_ev_made;
+    }
+    g_cur = g_calls;
   }
-  TLQ_CUDA_TRY(cudaEventRecord(g_ev[i], st));
-  if (i == TLQ_N_STAGES) g_ev_valid = true;
+  if (g_cur < 0) return TLQ_OK;
+  TLQ_CUDA_TRY(cudaEventRecord(g_ev[g_cur][i], st));
+  if (i == TLQ_N_STAGES) { ++g_calls; g_cur = -1; }
   return TLQ_OK;
 }
 
@@ -303,17 +312,23 @@ int tlq_read_status(const void* workspace, void* stream) {
 
 int tlq_stage_timing_enable(int on) {
   g_timing_on = on != 0;
-  g_ev_valid = false;
+  g_calls = 0;
+  g_cur = -1;
   return TLQ_OK;
 }
 
-int tlq_stage_timing_read(float* ms_out) {
-  if (ms_out == nullptr) return TLQ_ERR_INVALID_ARG;
-  if (!g_timing_on || !g_ev_valid) return TLQ_ERR_INVALID_ARG;
-  if (cudaEventSynchronize(g_ev[TLQ_N_STAGES]) != cudaSuccess) return TLQ_ERR_CUDA;
-  for (int i = 0; i < TLQ_N_STAGES; ++i)
-    if (cudaEventElapsedTime(&ms_out[i], g_ev[i], g_ev[i + 1]) != cudaSuccess) return TLQ_ERR_CUDA;
-  return TLQ_OK;
+int tlq_stage_timing_drain(float* ms_out, int max_calls) {
+  if (ms_out == nullptr || max_calls < 0) return TLQ_ERR_INVALID_ARG;
+  if (!g_timing_on) return TLQ_ERR_INVALID_ARG;
+  const int n = g_calls < max_calls ? g_calls : max_calls;
+  for (int c = 0; c < n; ++c) {
+    if (cudaEventSynchronize(g_ev[c][TLQ_N_STAGES]) != cudaSuccess) return TLQ_ERR_CUDA;
+    for (int i = 0; i < TLQ_N_STAGES; ++i)
+      if (cudaEventElapsedTime(&ms_out[c * TLQ_N_STAGES + i], g_ev[c][i], g_ev[c][i + 1]) != cudaSuccess)
+        return TLQ_ERR_CUDA;
+  }
+  g_calls = 0;
+  return n;
 }
 
 }  // extern "C"

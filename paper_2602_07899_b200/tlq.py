@@ -30,7 +30,7 @@ EXPORTS = (
     "tlq_status_string", "tlq_version", "tlq_token_importance", "tlq_scale_candidates_workspace_bytes",
     "tlq_scale_candidates", "tlq_quantize_weights", "tlq_scale_search_workspace_bytes", "tlq_scale_search_layer",
     "tlq_apply_layer_workspace_bytes", "tlq_apply_layer", "tlq_read_status", "tlq_stage_timing_enable",
-    "tlq_stage_timing_read", "tlq_kernel_launch_count",
+    "tlq_stage_timing_drain", "tlq_kernel_launch_count",
 )
 
 
@@ -79,9 +79,9 @@ def _load() -> ctypes.CDLL:
     lib.tlq_apply_layer.argtypes = [vp, i64, i64, vp, i64, vp, vp, cfgp, vp, sz, vp, vp, vp, vp, vp]
     lib.tlq_read_status.argtypes = [vp, vp]
     lib.tlq_stage_timing_enable.argtypes = [i32]
-    lib.tlq_stage_timing_read.argtypes = [ctypes.POINTER(ctypes.c_float)]
+    lib.tlq_stage_timing_drain.argtypes = [ctypes.POINTER(ctypes.c_float), i32]
     for fn in ("tlq_token_importance", "tlq_scale_candidates", "tlq_quantize_weights", "tlq_scale_search_layer",
-               "tlq_apply_layer", "tlq_read_status", "tlq_stage_timing_enable", "tlq_stage_timing_read"):
+               "tlq_apply_layer", "tlq_read_status", "tlq_stage_timing_enable", "tlq_stage_timing_drain"):
         getattr(lib, fn).restype = i32
     return lib
 
@@ -235,10 +235,13 @@ def tlq_stage_timing_enable(on: bool) -> None:
     _check(lib.tlq_stage_timing_enable(1 if on else 0), "tlq_stage_timing_enable")
 
 
-def tlq_stage_timing_read():
-    arr = (ctypes.c_float * N_STAGES)()
-    _check(lib.tlq_stage_timing_read(arr), "tlq_stage_timing_read")
-    return [float(v) for v in arr]
+def tlq_stage_timing_drain(max_calls: int = 512):
+    """-> list of per-call [stats, fakequant, gemm, reduce] milliseconds, oldest call first."""
+    arr = (ctypes.c_float * (N_STAGES * max_calls))()
+    n = lib.tlq_stage_timing_drain(arr, max_calls)
+    if n < 0:
+        raise TlqError(n, "tlq_stage_timing_drain")
+    return [[float(arr[c * N_STAGES + i]) for i in range(N_STAGES)] for c in range(n)]
 
 
 def tlq_kernel_launch_count() -> int:

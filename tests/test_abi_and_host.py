@@ -93,7 +93,7 @@ def test_host_validation_error_codes(tlq):
     assert L.tlq_token_importance(a, 0, 1, 4, 8, 0, 1.5, a, None, None) == tlq.ERR_INVALID_ARG
     assert L.tlq_read_status(None, None) == tlq.ERR_INVALID_ARG
     arr = (ctypes.c_float * 4)()
-    assert L.tlq_stage_timing_read(arr) == tlq.ERR_INVALID_ARG      # timing never enabled
+    assert L.tlq_stage_timing_drain(arr, 1) == tlq.ERR_INVALID_ARG  # timing never enabled
 
 
 def test_oracle_never_imports_the_cuda_path():
