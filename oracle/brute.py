@@ -73,7 +73,7 @@ def search(x_bits, w_bits, w_imp, group: int, n_grid: int, bits: int = 4, mode: 
                     zero = min(max(-round_half_even(f32(min(p) / step)), 0), qmax)
                     for j, c in enumerate(range(g0, g0 + group)):
                         q = min(max(round_half_even(f32(p[j] / step)) + zero, 0), qmax)
-                        w_hat[o][c] = f32(f32((q - zero) * step) / s[c])
+                        w_hat[o][c] = f32(f32((q - zero) * step) * f32(1.0 / s[c]))
             for i in range(n):
                 for o in range(c2):
                     y_q[i][o] = sum(w_hat[o][c] * x[i][c] for c in range(c1))

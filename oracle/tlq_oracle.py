@@ -22,8 +22,8 @@ What the paper fixes, and where each function comes from:
 Contract points (where floating point decides an integer the decision is taken in binary32, the
 precision of the CUDA kernels; everything else is float64): the product scale*w (exact in binary32
 for bf16 factors), the group range, the step, the zero-point quotient, the code quotient, the
-dequantized value and the division by the scale.  They are written with numpy float32 arrays, one
-IEEE operation per statement.
+dequantized value, the reciprocal of the scale and the product with it.  They are written with
+numpy float32 arrays, one IEEE operation per statement.
 
 Readings of silent points (the grid r_k = k/K, bf16 storage of the scale, half-to-even rounding,
 floors on degenerate statistics, loss normalisation by C2 * sum(w)) are listed in the design notes.
@@ -122,8 +122,9 @@ def quantize_weights_group_asym(w_bits: np.ndarray, s: np.ndarray | None, group:
     of one output row share a step and an integer zero-point.
 
     Returns (codes uint8 [C2,C1], step float32 [C2,C1/G], zero int32 [C2,C1/G], w_hat float32 [C2,C1])
-    where w_hat = dequant / scale is the weight the quantized layer effectively applies to the
-    unscaled activations (Sec. 2.2 smoothing identity).
+    where w_hat = dequant * (1/scale) is the weight the quantized layer effectively applies to the
+    unscaled activations (Sec. 2.2 smoothing identity); 1/scale is the same binary32 reciprocal that
+    smooths the activations in quantize_activations_token_sym.
     """
     w = bf16_to_f64(w_bits)
     c2, c1 = w.shape
@@ -143,7 +144,8 @@ def quantize_weights_group_asym(w_bits: np.ndarray, s: np.ndarray | None, group:
     cq = (pg / step[:, :, None]).astype(F32)              # binary32 division
     codes = np.clip(np.rint(cq).astype(np.int64) + zero[:, :, None], 0, qmax)
     dq = ((codes - zero[:, :, None]).astype(F32) * step[:, :, None]).astype(F32)   # binary32 product
-    w_hat = (dq.reshape(c2, c1) / sv.astype(F32)[None, :]).astype(F32)             # binary32 division
+    rs = (F32(1.0) / sv.astype(F32)).astype(F32)                                   # binary32 reciprocal of the scale
+    w_hat = (dq.reshape(c2, c1) * rs[None, :]).astype(F32)                         # binary32 product
     return codes.reshape(c2, c1).astype(np.uint8), step, zero, w_hat
 
 

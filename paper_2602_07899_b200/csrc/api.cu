@@ -210,7 +210,7 @@ int tlq_quantize_weights(const void* W, const void* s, int64_t C2, int64_t C1, c
   const uint16_t* Wb = reinterpret_cast<const uint16_t*>(W);
   const uint16_t* sb = reinterpret_cast<const uint16_t*>(s);
   if (cfg->mode == TLQ_W4A16_ASYM_GROUP)
-    return launch_fakequant_group(Wb, sb, 1, C2, C1, cfg->group_size, cfg->w_bits, reinterpret_cast<uint16_t*>(dW_out),
+    return launch_fakequant_group(Wb, sb, nullptr, 1, C2, C1, cfg->group_size, cfg->w_bits, reinterpret_cast<uint16_t*>(dW_out),
                                   codes, steps, zeros, st);
   if (dW_out != nullptr || codes == nullptr || steps == nullptr) return TLQ_ERR_INVALID_ARG;
   return launch_fakequant_rows_i8(Wb, sb, 1, C2, C1, reinterpret_cast<int8_t*>(codes), steps, st);
@@ -248,7 +248,7 @@ int tlq_scale_search_layer(const void* X, int64_t N, int64_t C1, const void* W, 
                                st)) != TLQ_OK)
     return rc;
   if ((rc = timing_mark(1, st)) != TLQ_OK) return rc;
-  if ((rc = launch_fakequant_group(Wb, L.s, K, C2, C1, cfg->group_size, cfg->w_bits, L.dW, nullptr, nullptr, nullptr,
+  if ((rc = launch_fakequant_group(Wb, L.s, L.rs, K, C2, C1, cfg->group_size, cfg->w_bits, L.dW, nullptr, nullptr, nullptr,
                                    st)) != TLQ_OK)
     return rc;
   if ((rc = timing_mark(2, st)) != TLQ_OK) return rc;
@@ -293,7 +293,7 @@ int tlq_apply_layer(const void* X, int64_t N, int64_t C1, const void* W, int64_t
   const uint16_t* Xb = reinterpret_cast<const uint16_t*>(X);
   const uint16_t* Wb = reinterpret_cast<const uint16_t*>(W);
   TLQ_CUDA_TRY(cudaMemsetAsync(hdr, 0, sizeof(WorkspaceHeader), st));
-  if ((rc = launch_fakequant_group(Wb, reinterpret_cast<const uint16_t*>(s), 1, C2, C1, cfg->group_size, cfg->w_bits,
+  if ((rc = launch_fakequant_group(Wb, reinterpret_cast<const uint16_t*>(s), nullptr, 1, C2, C1, cfg->group_size, cfg->w_bits,
                                    dW, codes, steps, zeros, st)) != TLQ_OK)
     return rc;
   return launch_apply_gemm_bf16(Xb, Wb, dW, reinterpret_cast<const uint16_t*>(bias), N, C1, C2,

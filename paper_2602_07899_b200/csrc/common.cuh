@@ -83,7 +83,8 @@ int launch_scale_table(const double* partials, int64_t chunks, int64_t N, int64_
                        cudaStream_t st);
 
 // fakequant.cu
-int launch_fakequant_group(const uint16_t* W, const uint16_t* s /*[K,C1] or null*/, int K, int64_t C2, int64_t C1,
+int launch_fakequant_group(const uint16_t* W, const uint16_t* s /*[K,C1] or null*/, const float* rs /*[K,C1] or null: 1/s*/,
+                           int K, int64_t C2, int64_t C1,
                            int group, int w_bits, uint16_t* dW /*[K,C2,C1] or null*/, uint8_t* codes, float* steps,
                            int32_t* zeros, cudaStream_t st);
 int launch_fakequant_rows_i8(const uint16_t* W, const uint16_t* s /*[K,C1] or null*/, int K, int64_t C2, int64_t C1,

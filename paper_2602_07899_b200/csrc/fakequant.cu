@@ -1,66 +1,131 @@
 // Fake-quantization kernels: Q_w(W * scale) for the group-wise asymmetric setting and the int8
 // symmetric row / token quantizers (paper Sec. 2.2 quantizer; Sec. 3.2.1 f_q).
 //
-// All are HBM-bound streaming kernels: a tile of the bf16 source is staged once in shared memory
-// and re-used for every scale candidate, so the source is read once and each candidate's operand
-// is written once.  Where floating point decides an integer (step, zero-point, code) the operation
-// is a single IEEE binary32 operation written with the *_rn intrinsics, so no contraction or
-// approximate division can change a code.
+// All are streaming kernels whose floor is HBM bandwidth: a tile of the bf16 source is staged once
+// in shared memory and re-used for every scale candidate, so the source is read once and each
+// candidate's operand is written once.  The arithmetic is kept off the slow conversion / reciprocal
+// unit: rounding to an integer is the add-and-subtract of 1.5*2^23 (exact round-half-even in
+// binary32 for |x| < 2^22), clamping stays in floating point, int8 codes are read out of the low
+// mantissa bits, and the per-element quotient value/step is taken as value * (1/step) with an exact
+// IEEE division only when the product lies so close to a rounding tie that the two could round
+// differently.  The integer produced is therefore always rint(fl32(value / step)), the contract the
+// CPU reference uses, at a fraction of the instruction count.
 #include "common.cuh"
 
 namespace tlq {
 
+namespace {
+
+constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23
+
+// rint(x) for |x| <= 2^21 without a conversion instruction.
+__device__ __forceinline__ float round_magic(float x) { return __fsub_rn(__fadd_rn(x, kMagic), kMagic); }
+
+// rint(fl32(v / step)) given inv = fl32(1 / step).
+// fl32(v * inv) is within |q| * 1.8e-7 of the true quotient and so is fl32(v / step); for |q| < 1024
+// that is below 2.5e-4, so when the product is farther than that from a tie both round to the same
+// integer.  For |q| >= 1024 every caller clamps to a range inside (-1024, 1024), where the integer
+// is saturated whichever way the quotient rounds.
+__device__ __forceinline__ float quotient_rint(float v, float step, float inv) {
+  float q = __fmul_rn(v, inv);
+  q = fminf(fmaxf(q, -2097152.0f), 2097152.0f);
+  float r = round_magic(q);
+  if (fabsf(__fsub_rn(q, r)) > 0.49975f && fabsf(q) < 1024.0f) {
+    const float exact = __fdiv_rn(v, step);
+    r = round_magic(exact);
+  }
+  return r;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+}  // namespace
+
 // ------------------------------------------------------------------------------------------------
 // Group-wise asymmetric weights (W4A16 and other widths).
-// Tile: kGqRows x 512 channels; a thread owns 8 consecutive channels, 64 threads span the 512
-// channels of one row, so one pass of the 256-thread CTA covers 4 rows.  A group of g channels is
-// g/8 adjacent lanes of one warp: min/max go through xor-shuffles.
+// Tile: kGqRows x 512 channels.  A thread owns 16 consecutive channels, a warp spans the 512 channels
+// of one row, the 8 warps of the CTA take 8 rows per pass.  A group of g channels is g/16 adjacent
+// lanes: min/max go through xor-shuffles.  grid.z splits the candidates when the matrix alone
+// would not fill the machine.
 // ------------------------------------------------------------------------------------------------
-constexpr int kGqRows = 16;
+constexpr int kGqRows = 32;
 constexpr int kGqCols = 512;
 constexpr int kGqThreads = 256;
 
 __global__ void __launch_bounds__(kGqThreads)
-fakequant_group_kernel(const uint16_t* __restrict__ W, const uint16_t* __restrict__ s_tab, int K, int64_t C2,
-                       int64_t C1, int group, int qmax, uint16_t* __restrict__ dW, uint8_t* __restrict__ codes,
-                       float* __restrict__ steps, int32_t* __restrict__ zeros) {
+fakequant_group_kernel(const uint16_t* __restrict__ W, const uint16_t* __restrict__ s_tab,
+                       const float* __restrict__ rs_tab, int K, int k_per_cta, int64_t C2, int64_t C1, int group,
+                       int qmax, uint16_t* __restrict__ dW, uint8_t* __restrict__ codes, float* __restrict__ steps,
+                       int32_t* __restrict__ zeros) {
   __shared__ uint4 tile[kGqRows][kGqCols / 8];
-  const int t = threadIdx.x;
-  const int col8 = t & 63;          // which 8-channel packet of the 512-wide tile
-  const int rsub = t >> 6;          // 0..3
-  const int64_t c0 = (int64_t)blockIdx.x * kGqCols + col8 * 8;
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int64_t c0 = (int64_t)blockIdx.x * kGqCols + lane * 16;
   const int64_t row0 = (int64_t)blockIdx.y * kGqRows;
-  const bool col_ok = c0 < C1;
-  const int lanes_per_group = group >> 3;
+  const bool col_ok = c0 < C1;                    // C1 % 16 == 0 is guaranteed by the group sizes
+  const int lanes_per_group = group >> 4;
   const float qmax_f = (float)qmax;
   const int64_t ngroups = C1 / group;
+  const int k_begin = blockIdx.z * k_per_cta;
+  const int k_end = min(K, k_begin + k_per_cta);
 
   // stage the W tile (zeros outside the matrix)
 #pragma unroll
-  for (int p = 0; p < kGqRows / 4; ++p) {
-    const int r = p * 4 + rsub;
-    uint4 v = make_uint4(0, 0, 0, 0);
-    if (col_ok && row0 + r < C2) v = ld_nc_16(W + (row0 + r) * C1 + c0);
-    tile[r][col8] = v;
+  for (int p = 0; p < kGqRows / 8; ++p) {
+    const int r = p * 8 + warp;
+    uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0;
+    if (col_ok && row0 + r < C2) {
+      const uint16_t* src = W + (row0 + r) * C1 + c0;
+      v0 = ld_nc_16(src);
+      v1 = ld_nc_16(src + 8);
+    }
+    tile[r][lane * 2] = v0;
+    tile[r][lane * 2 + 1] = v1;
   }
   __syncthreads();
 
-  for (int k = 0; k < K; ++k) {
-    float sv[8];
+  for (int k = k_begin; k < k_end; ++k) {
+    float sv[16], rsv[16];
     if (s_tab != nullptr && col_ok) {
-      unpack8(*reinterpret_cast<const uint4*>(s_tab + (int64_t)k * C1 + c0), sv);
+      const uint16_t* sp = s_tab + (int64_t)k * C1 + c0;
+      float a[8], b[8];
+      unpack8(*reinterpret_cast<const uint4*>(sp), a);
+      unpack8(*reinterpret_cast<const uint4*>(sp + 8), b);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { sv[j] = a[j]; sv[8 + j] = b[j]; }
+      if (rs_tab != nullptr) {
+        const float4* rp = reinterpret_cast<const float4*>(rs_tab + (int64_t)k * C1 + c0);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float4 r4 = rp[j];
+          rsv[j * 4] = r4.x; rsv[j * 4 + 1] = r4.y; rsv[j * 4 + 2] = r4.z; rsv[j * 4 + 3] = r4.w;
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) rsv[j] = __fdiv_rn(1.0f, sv[j]);
+      }
     } else {
 #pragma unroll
-      for (int j = 0; j < 8; ++j) sv[j] = 1.0f;
+      for (int j = 0; j < 16; ++j) { sv[j] = 1.0f; rsv[j] = 1.0f; }
     }
+#pragma unroll 1
+    for (int p = 0; p < kGqRows / 8; ++p) {
+      const int r = p * 8 + warp;
+      float w[16], pr[16];
+      {
+        float a[8], b[8];
+        unpack8(tile[r][lane * 2], a);
+        unpack8(tile[r][lane * 2 + 1], b);
 #pragma unroll
-    for (int p = 0; p < kGqRows / 4; ++p) {
-      const int r = p * 4 + rsub;
-      float w[8], pr[8];
-      unpack8(tile[r][col8], w);
+        for (int j = 0; j < 8; ++j) { w[j] = a[j]; w[8 + j] = b[j]; }
+      }
       float mx, mn;
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
+      for (int j = 0; j < 16; ++j) {
         pr[j] = __fmul_rn(sv[j], w[j]);            // exact: 8-bit x 8-bit significands
         mx = (j == 0) ? pr[0] : fmaxf(mx, pr[j]);
         mn = (j == 0) ? pr[0] : fminf(mn, pr[j]);
@@ -69,28 +134,39 @@ fakequant_group_kernel(const uint16_t* __restrict__ W, const uint16_t* __restric
         mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
         mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, off));
       }
-      float range = fmaxf(__fsub_rn(mx, mn), TLQ_RANGE_FLOOR);
+      const float range = fmaxf(__fsub_rn(mx, mn), TLQ_RANGE_FLOOR);
       const float step = __fdiv_rn(range, qmax_f);
+      const float inv = __fdiv_rn(1.0f, step);
       int z = -__float2int_rn(__fdiv_rn(mn, step));
       z = min(max(z, 0), qmax);
-      uint32_t outw[4];
-      uint32_t qpack[2] = {0u, 0u};
+      const float zf = (float)z;
+      uint32_t outw[8];
+      uint32_t qpack[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        int q = __float2int_rn(__fdiv_rn(pr[j], step)) + z;
-        q = min(max(q, 0), qmax);
-        const float dq = __fmul_rn((float)(q - z), step);
-        const float w_hat = __fdiv_rn(dq, sv[j]);
-        const uint32_t b = float_to_bf16_bits(__fsub_rn(w[j], w_hat));
-        if (j & 1) outw[j >> 1] |= b << 16; else outw[j >> 1] = b;
-        qpack[j >> 2] |= (uint32_t)q << ((j & 3) * 8);
+      for (int j = 0; j < 16; j += 2) {
+        float d[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          float q = __fadd_rn(quotient_rint(pr[j + h], step, inv), zf);
+          q = fminf(fmaxf(q, 0.0f), qmax_f);
+          const float dq = __fmul_rn(__fsub_rn(q, zf), step);
+          const float w_hat = __fmul_rn(dq, rsv[j + h]);
+          d[h] = __fsub_rn(w[j + h], w_hat);
+          if (codes != nullptr)
+            qpack[(j + h) >> 2] |= (__float_as_uint(__fadd_rn(q, kMagic)) & 0xFFu) << (((j + h) & 3) * 8);
+        }
+        outw[j >> 1] = pack_bf16x2(d[0], d[1]);
       }
       const int64_t row = row0 + r;
       if (col_ok && row < C2) {
-        if (dW != nullptr)
-          *reinterpret_cast<uint4*>(dW + ((int64_t)k * C2 + row) * C1 + c0) = make_uint4(outw[0], outw[1], outw[2], outw[3]);
-        if (codes != nullptr) *reinterpret_cast<uint2*>(codes + row * C1 + c0) = make_uint2(qpack[0], qpack[1]);
-        if ((col8 % lanes_per_group) == 0) {
+        if (dW != nullptr) {
+          uint4* dst = reinterpret_cast<uint4*>(dW + ((int64_t)k * C2 + row) * C1 + c0);
+          dst[0] = make_uint4(outw[0], outw[1], outw[2], outw[3]);
+          dst[1] = make_uint4(outw[4], outw[5], outw[6], outw[7]);
+        }
+        if (codes != nullptr)
+          *reinterpret_cast<uint4*>(codes + row * C1 + c0) = make_uint4(qpack[0], qpack[1], qpack[2], qpack[3]);
+        if ((lane % lanes_per_group) == 0) {
           const int64_t g = c0 / group;
           if (steps != nullptr) steps[row * ngroups + g] = step;
           if (zeros != nullptr) zeros[row * ngroups + g] = z;
@@ -100,12 +176,18 @@ fakequant_group_kernel(const uint16_t* __restrict__ W, const uint16_t* __restric
   }
 }
 
-int launch_fakequant_group(const uint16_t* W, const uint16_t* s, int K, int64_t C2, int64_t C1, int group,
-                           int w_bits, uint16_t* dW, uint8_t* codes, float* steps, int32_t* zeros,
+int launch_fakequant_group(const uint16_t* W, const uint16_t* s, const float* rs, int K, int64_t C2, int64_t C1,
+                           int group, int w_bits, uint16_t* dW, uint8_t* codes, float* steps, int32_t* zeros,
                            cudaStream_t st) {
-  dim3 grid((unsigned)ceil_div(C1, kGqCols), (unsigned)ceil_div(C2, kGqRows));
-  fakequant_group_kernel<<<grid, kGqThreads, 0, st>>>(W, s, K, C2, C1, group, (1 << w_bits) - 1, dW, codes, steps,
-                                                     zeros);
+  const int64_t ctas = ceil_div(C1, kGqCols) * ceil_div(C2, kGqRows);
+  int64_t kchunks = ceil_div(148 * 6, ctas);        // aim for several CTAs per SM
+  if (kchunks > K) kchunks = K;
+  if (kchunks < 1) kchunks = 1;
+  const int k_per_cta = (int)ceil_div(K, kchunks);
+  kchunks = ceil_div(K, k_per_cta);
+  dim3 grid((unsigned)ceil_div(C1, kGqCols), (unsigned)ceil_div(C2, kGqRows), (unsigned)kchunks);
+  fakequant_group_kernel<<<grid, kGqThreads, 0, st>>>(W, s, rs, K, k_per_cta, C2, C1, group, (1 << w_bits) - 1, dW,
+                                                     codes, steps, zeros);
   return after_launch();
 }
 
@@ -158,8 +240,7 @@ quant_rows_i8_kernel(const uint16_t* __restrict__ src, const uint16_t* __restric
                      const float* __restrict__ rs_tab, int K, int64_t R, int64_t C1, int8_t* __restrict__ q,
                      float* __restrict__ step_out) {
   extern __shared__ uint4 row_smem[];      // C1/8 packets
-  __shared__ float warp_max[kRowThreads / 32];
-  __shared__ float row_step;
+  __shared__ float warp_max[2][kRowThreads / 32];
   const int t = threadIdx.x;
   for (int64_t row = blockIdx.x; row < R; row += gridDim.x) {
     __syncthreads();
@@ -177,18 +258,15 @@ quant_rows_i8_kernel(const uint16_t* __restrict__ src, const uint16_t* __restric
       }
 #pragma unroll
       for (int off = 16; off > 0; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, off));
-      if ((t & 31) == 0) warp_max[t >> 5] = amax;
+      float* wm = warp_max[k & 1];          // double-buffered: one barrier per candidate
+      if ((t & 31) == 0) wm[t >> 5] = amax;
       __syncthreads();
-      if (t == 0) {
-        float m = warp_max[0];
+      float m = wm[0];
 #pragma unroll
-        for (int w = 1; w < kRowThreads / 32; ++w) m = fmaxf(m, warp_max[w]);
-        const float st = __fdiv_rn(fmaxf(m, TLQ_RANGE_FLOOR), 127.0f);
-        row_step = st;
-        step_out[(int64_t)k * R + row] = st;
-      }
-      __syncthreads();
-      const float st = row_step;
+      for (int w = 1; w < kRowThreads / 32; ++w) m = fmaxf(m, wm[w]);
+      const float st = __fdiv_rn(fmaxf(m, TLQ_RANGE_FLOOR), 127.0f);
+      const float inv = __fdiv_rn(1.0f, st);
+      if (t == 0) step_out[(int64_t)k * R + row] = st;
       int8_t* out = q + ((int64_t)k * R + row) * C1;
       for (int64_t c = (int64_t)t * 16; c < C1; c += kRowThreads * 16) {
         float v[16];
@@ -196,9 +274,9 @@ quant_rows_i8_kernel(const uint16_t* __restrict__ src, const uint16_t* __restric
         uint32_t pk[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-          int qi = __float2int_rn(__fdiv_rn(v[j], st));
-          qi = min(max(qi, -128), 127);
-          pk[j >> 2] |= ((uint32_t)qi & 0xFFu) << ((j & 3) * 8);
+          float qi = quotient_rint(v[j], st, inv);
+          qi = fminf(fmaxf(qi, -128.0f), 127.0f);
+          pk[j >> 2] |= (__float_as_uint(__fadd_rn(qi, kMagic)) & 0xFFu) << ((j & 3) * 8);
         }
         *reinterpret_cast<uint4*>(out + c) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
       }

@@ -220,16 +220,16 @@ def test_apply_layer(tlq):
     assert np.array_equal(out["zeros"].cpu().numpy(), zero)
     yq = out["Yq"].float().cpu().numpy().astype(np.float64)
     # bf16 output rounding (half an ulp = 2^-9 relative, doubled for slack) plus the bf16 rounding of the
-    # delta-weight operand, which perturbs a token's output by a fraction of that token's rms output error
+    # delta-weight operand, which perturbs an output by a few 1e-3 of the token's rms output error (4 sigma and per-output spread: 2e-2)
     rms_e = np.sqrt(ref["per_token"][ref["best"]] / 328.0)[:, None]
     err = np.abs(yq - yq_ref)
-    assert np.all(err <= 2.0 ** -8 * np.abs(yq_ref) + 5e-3 * rms_e + 1e-6)
+    assert np.all(err <= 2.0 ** -8 * np.abs(yq_ref) + 2e-2 * rms_e + 1e-6)
     # without scale and bias
     out0 = tlq.tlq_apply_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), None, None, tlq.config(), want_codes=False)
     y0_ref, _ = orc.apply_layer(xb, wb, None, None, "w4a16", 128)
     y0 = out0["Yq"].float().cpu().numpy().astype(np.float64)
     rms0 = np.sqrt(ref["per_token"][0] / 328.0)[:, None]
-    assert np.all(np.abs(y0 - y0_ref) <= 2.0 ** -8 * np.abs(y0_ref) + 5e-3 * rms0 + 1e-6)
+    assert np.all(np.abs(y0 - y0_ref) <= 2.0 ** -8 * np.abs(y0_ref) + 2e-2 * rms0 + 1e-6)
 
 
 def test_device_errors_are_reported_not_raised_as_faults(tlq):
