@@ -121,6 +121,14 @@ int tlq_quantize_weights(const void* W, const void* s, int64_t C2, int64_t C1, c
                          uint8_t* codes, float* steps, int32_t* zeros, void* dW_out, void* stream);
 
 /*
+ * Quantize the smoothed activations for ONE scale vector: Q_a(x / scale), per-token symmetric int8
+ * (Sec. 2.2 first two equations; Sec. 3.2.1 f_q).  W8A8 mode only.
+ *   X [N,C1] bf16; s [C1] bf16 or NULL (= ones); codes [N,C1] int8; steps [N] fp32.
+ */
+int tlq_quantize_activations(const void* X, const void* s, int64_t N, int64_t C1, const tlq_config* cfg,
+                             int8_t* codes, float* steps, void* stream);
+
+/*
  * The layer-wise search (Sec. 3.2.1): for k in [0,K): loss[k] = sum_n w_n e_{k,n} / (C2 * sum_n w_n),
  * e_{k,n} = || f_fp(x_n) - f_q(x_n; scale_k) ||_2^2; best_idx = argmin (lowest index on ties).
  *   X [N,C1] bf16, W [C2,C1] bf16, w_imp [N] fp32 >= 0 or NULL (uniform),

@@ -72,20 +72,23 @@ struct SearchLayout {
   float* t;
   size_t bytes;
   GemmPlan plan;
+  int64_t ptab_slices;   // per-candidate slices of the per-token table (column tiles, x2 for W8A8)
 };
 
 SearchLayout carve_search(void* ws, int64_t N, int64_t C1, int64_t C2, const tlq_config* cfg) {
   SearchLayout L{};
   const int K = cfg->n_grid;
   Carver c(ws);
-  L.plan = plan_search_gemm(N, C1, C2, K);
+  const bool i8 = cfg->mode == TLQ_W8A8_SYM;
+  L.plan = i8 ? plan_search_gemm_i8(N, C1, C2, K) : plan_search_gemm(N, C1, C2, K);
+  L.ptab_slices = L.plan.otiles * (i8 ? 2 : 1);
   L.hdr = c.take<WorkspaceHeader>(1);
   L.stat_partials = c.take<double>((size_t)stats_row_chunks(N) * C1);
   L.x_stat = c.take<double>((size_t)C1);
   L.s = c.take<uint16_t>((size_t)K * C1);
   L.rs = c.take<float>((size_t)K * C1);
   L.partials = c.take<float>((size_t)K * L.plan.partials_per_k);
-  L.ptab = c.take<float>((size_t)K * L.plan.otiles * L.plan.n_pad);
+  L.ptab = c.take<float>((size_t)K * L.ptab_slices * L.plan.n_pad);
   if (cfg->mode == TLQ_W4A16_ASYM_GROUP) {
     L.dW = c.take<uint16_t>((size_t)K * C2 * C1, 1024);
   } else {
@@ -216,6 +219,20 @@ int tlq_quantize_weights(const void* W, const void* s, int64_t C2, int64_t C1, c
   return launch_fakequant_rows_i8(Wb, sb, 1, C2, C1, reinterpret_cast<int8_t*>(codes), steps, st);
 }
 
+int tlq_quantize_activations(const void* X, const void* s, int64_t N, int64_t C1, const tlq_config* cfg, int8_t* codes,
+                             float* steps, void* stream) {
+  if (X == nullptr || codes == nullptr || steps == nullptr) return TLQ_ERR_INVALID_ARG;
+  if (N < 1) return TLQ_ERR_SHAPE;
+  int rc = check_cfg(cfg, C1);
+  if (rc != TLQ_OK) return rc;
+  if (cfg->mode != TLQ_W8A8_SYM) return TLQ_ERR_UNSUPPORTED;
+  if (!aligned16(X) || (s != nullptr && !aligned16(s)) || !aligned16(codes)) return TLQ_ERR_ALIGN;
+  rc = have_device();
+  if (rc != TLQ_OK) return rc;
+  return launch_actquant_i8(reinterpret_cast<const uint16_t*>(X), reinterpret_cast<const uint16_t*>(s), nullptr, 1, N,
+                            C1, codes, steps, reinterpret_cast<cudaStream_t>(stream));
+}
+
 size_t tlq_scale_search_workspace_bytes(int64_t N, int64_t C1, int64_t C2, const tlq_config* cfg) {
   if (N < 1 || C2 < 1 || check_cfg(cfg, C1) != TLQ_OK) return 0;
   return carve_search(nullptr, N, C1, C2, cfg).bytes;
@@ -231,7 +248,6 @@ int tlq_scale_search_layer(const void* X, int64_t N, int64_t C1, const void* W, 
   if (rc != TLQ_OK) return rc;
   if (cfg->stat_mode == TLQ_STAT_MASKED_MAX && mask == nullptr) return TLQ_ERR_INVALID_ARG;
   if (!aligned16(X) || !aligned16(W) || !aligned16(workspace)) return TLQ_ERR_ALIGN;
-  if (cfg->mode == TLQ_W8A8_SYM) return TLQ_ERR_UNSUPPORTED;
   SearchLayout L = carve_search(workspace, N, C1, C2, cfg);
   if (workspace_bytes < L.bytes) return TLQ_ERR_WORKSPACE;
   rc = have_device();
@@ -248,28 +264,61 @@ int tlq_scale_search_layer(const void* X, int64_t N, int64_t C1, const void* W, 
                                st)) != TLQ_OK)
     return rc;
   if ((rc = timing_mark(1, st)) != TLQ_OK) return rc;
-  if ((rc = launch_fakequant_group(Wb, L.s, L.rs, K, C2, C1, cfg->group_size, cfg->w_bits, L.dW, nullptr, nullptr, nullptr,
-                                   st)) != TLQ_OK)
-    return rc;
-  if ((rc = timing_mark(2, st)) != TLQ_OK) return rc;
   float* ptab = (per_token_err != nullptr) ? L.ptab : nullptr;
-  if ((rc = launch_search_gemm_bf16(Xb, L.dW, w_imp, L.plan, L.partials, ptab, L.hdr, st)) != TLQ_OK) return rc;
+  if (cfg->mode == TLQ_W4A16_ASYM_GROUP) {
+    if ((rc = launch_fakequant_group(Wb, L.s, L.rs, K, C2, C1, cfg->group_size, cfg->w_bits, L.dW, nullptr, nullptr,
+                                     nullptr, st)) != TLQ_OK)
+      return rc;
+    if ((rc = timing_mark(2, st)) != TLQ_OK) return rc;
+    if ((rc = launch_search_gemm_bf16(Xb, L.dW, w_imp, L.plan, L.partials, ptab, L.hdr, st)) != TLQ_OK) return rc;
+  } else {
+    if ((rc = launch_fakequant_rows_i8(Wb, L.s, K, C2, C1, L.Wq, L.u, st)) != TLQ_OK) return rc;
+    if ((rc = launch_actquant_i8(Xb, nullptr, L.rs, K, N, C1, L.Xq, L.t, st)) != TLQ_OK) return rc;
+    if ((rc = timing_mark(2, st)) != TLQ_OK) return rc;
+    if ((rc = launch_search_gemm_i8(Xb, Wb, L.Xq, L.Wq, L.t, L.u, w_imp, L.plan, L.partials, ptab, L.hdr, st)) !=
+        TLQ_OK)
+      return rc;
+  }
   if ((rc = timing_mark(3, st)) != TLQ_OK) return rc;
   if ((rc = launch_loss_reduce(L.partials, L.plan.partials_per_k, K, w_imp, N, C2, L.s, C1, L.hdr, losses, best_idx,
                                reinterpret_cast<uint16_t*>(s_best), st)) != TLQ_OK)
     return rc;
   if (per_token_err != nullptr)
-    if ((rc = launch_per_token_reduce(L.ptab, K, L.plan.otiles, L.plan.n_pad, N, per_token_err, st)) != TLQ_OK)
+    if ((rc = launch_per_token_reduce(L.ptab, K, L.ptab_slices, L.plan.n_pad, N, per_token_err, st)) != TLQ_OK)
       return rc;
   return timing_mark(4, st);
 }
 
+namespace {
+struct ApplyLayout {
+  WorkspaceHeader* hdr;
+  uint16_t* dW;
+  int8_t* Wq;
+  float* u;
+  int8_t* Xq;
+  float* t;
+  size_t bytes;
+};
+ApplyLayout carve_apply(void* ws, int64_t N, int64_t C1, int64_t C2, const tlq_config* cfg) {
+  ApplyLayout L{};
+  Carver c(ws);
+  L.hdr = c.take<WorkspaceHeader>(1);
+  if (cfg->mode == TLQ_W4A16_ASYM_GROUP) {
+    L.dW = c.take<uint16_t>((size_t)C2 * C1, 1024);
+  } else {
+    L.Wq = c.take<int8_t>((size_t)C2 * C1, 1024);
+    L.u = c.take<float>((size_t)C2);
+    L.Xq = c.take<int8_t>((size_t)N * C1, 1024);
+    L.t = c.take<float>((size_t)N);
+  }
+  L.bytes = align_up(c.off, 256);
+  return L;
+}
+}  // namespace
+
 size_t tlq_apply_layer_workspace_bytes(int64_t N, int64_t C1, int64_t C2, const tlq_config* cfg) {
   if (N < 1 || C2 < 1 || check_cfg(cfg, C1) != TLQ_OK) return 0;
-  Carver c(nullptr);
-  c.take<WorkspaceHeader>(1);
-  c.take<uint16_t>((size_t)C2 * C1, 1024);
-  return align_up(c.off, 256);
+  return carve_apply(nullptr, N, C1, C2, cfg).bytes;
 }
 
 int tlq_apply_layer(const void* X, int64_t N, int64_t C1, const void* W, int64_t C2, const void* s, const void* bias,
@@ -282,22 +331,27 @@ int tlq_apply_layer(const void* X, int64_t N, int64_t C1, const void* W, int64_t
   if (!aligned16(X) || !aligned16(W) || !aligned16(workspace) || !aligned16(Yq) || (s != nullptr && !aligned16(s)) ||
       (codes != nullptr && !aligned16(codes)))
     return TLQ_ERR_ALIGN;
-  if (cfg->mode == TLQ_W8A8_SYM) return TLQ_ERR_UNSUPPORTED;
-  if (workspace_bytes < tlq_apply_layer_workspace_bytes(N, C1, C2, cfg)) return TLQ_ERR_WORKSPACE;
+  ApplyLayout L = carve_apply(workspace, N, C1, C2, cfg);
+  if (workspace_bytes < L.bytes) return TLQ_ERR_WORKSPACE;
   rc = have_device();
   if (rc != TLQ_OK) return rc;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  Carver c(workspace);
-  WorkspaceHeader* hdr = c.take<WorkspaceHeader>(1);
-  uint16_t* dW = c.take<uint16_t>((size_t)C2 * C1, 1024);
   const uint16_t* Xb = reinterpret_cast<const uint16_t*>(X);
   const uint16_t* Wb = reinterpret_cast<const uint16_t*>(W);
-  TLQ_CUDA_TRY(cudaMemsetAsync(hdr, 0, sizeof(WorkspaceHeader), st));
-  if ((rc = launch_fakequant_group(Wb, reinterpret_cast<const uint16_t*>(s), nullptr, 1, C2, C1, cfg->group_size, cfg->w_bits,
-                                   dW, codes, steps, zeros, st)) != TLQ_OK)
-    return rc;
-  return launch_apply_gemm_bf16(Xb, Wb, dW, reinterpret_cast<const uint16_t*>(bias), N, C1, C2,
-                                reinterpret_cast<uint16_t*>(Yq), hdr, st);
+  const uint16_t* sb = reinterpret_cast<const uint16_t*>(s);
+  const uint16_t* bb = reinterpret_cast<const uint16_t*>(bias);
+  TLQ_CUDA_TRY(cudaMemsetAsync(L.hdr, 0, sizeof(WorkspaceHeader), st));
+  if (cfg->mode == TLQ_W4A16_ASYM_GROUP) {
+    if ((rc = launch_fakequant_group(Wb, sb, nullptr, 1, C2, C1, cfg->group_size, cfg->w_bits, L.dW, codes, steps,
+                                     zeros, st)) != TLQ_OK)
+      return rc;
+    return launch_apply_gemm_bf16(Xb, Wb, L.dW, bb, N, C1, C2, reinterpret_cast<uint16_t*>(Yq), L.hdr, st);
+  }
+  if ((rc = launch_fakequant_rows_i8(Wb, sb, 1, C2, C1, L.Wq, L.u, st)) != TLQ_OK) return rc;
+  if ((rc = launch_actquant_i8(Xb, sb, nullptr, 1, N, C1, L.Xq, L.t, st)) != TLQ_OK) return rc;
+  if (codes != nullptr) TLQ_CUDA_TRY(cudaMemcpyAsync(codes, L.Wq, (size_t)C2 * C1, cudaMemcpyDeviceToDevice, st));
+  if (steps != nullptr) TLQ_CUDA_TRY(cudaMemcpyAsync(steps, L.u, (size_t)C2 * sizeof(float), cudaMemcpyDeviceToDevice, st));
+  return launch_apply_gemm_i8(L.Xq, L.Wq, L.t, L.u, bb, N, C1, C2, reinterpret_cast<uint16_t*>(Yq), L.hdr, st);
 }
 
 int tlq_read_status(const void* workspace, void* stream) {

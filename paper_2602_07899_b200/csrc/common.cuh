@@ -89,7 +89,8 @@ int launch_fakequant_group(const uint16_t* W, const uint16_t* s /*[K,C1] or null
                            int32_t* zeros, cudaStream_t st);
 int launch_fakequant_rows_i8(const uint16_t* W, const uint16_t* s /*[K,C1] or null*/, int K, int64_t C2, int64_t C1,
                              int8_t* q /*[K,C2,C1]*/, float* u /*[K,C2]*/, cudaStream_t st);
-int launch_actquant_i8(const uint16_t* X, const float* rs /*[K,C1] or null*/, int K, int64_t N, int64_t C1,
+// activations: x * (1/s); give the reciprocal table rs [K,C1], or a bf16 scale s [K,C1] to invert on the fly, or neither
+int launch_actquant_i8(const uint16_t* X, const uint16_t* s, const float* rs, int K, int64_t N, int64_t C1,
                        int8_t* q /*[K,N,C1]*/, float* t /*[K,N]*/, cudaStream_t st);
 
 // importance.cu
@@ -119,5 +120,15 @@ int launch_search_gemm_bf16(const uint16_t* X, const uint16_t* dW, const float* 
 // Apply: Yq[N,C2] = X W^T - X dW^T (+bias), bf16 out
 int launch_apply_gemm_bf16(const uint16_t* X, const uint16_t* W, const uint16_t* dW, const uint16_t* bias,
                            int64_t N, int64_t C1, int64_t C2, uint16_t* Yq, WorkspaceHeader* hdr, cudaStream_t st);
+
+// search_gemm_i8.cu
+GemmPlan plan_search_gemm_i8(int64_t N, int64_t C1, int64_t C2, int K);   // partials_per_k = mtiles*otiles*8
+// W8A8 search: partials[K][mtiles*otiles*8] (+ ptab[K][otiles*2][n_pad] if non-null)
+int launch_search_gemm_i8(const uint16_t* X, const uint16_t* W, const int8_t* Xq, const int8_t* Wq, const float* t,
+                          const float* u, const float* w_imp, const GemmPlan& plan, float* partials, float* ptab,
+                          WorkspaceHeader* hdr, cudaStream_t st);
+// Apply: Yq[N,C2] = t[n] * u[o] * (Xq Wq^T) (+bias), bf16 out
+int launch_apply_gemm_i8(const int8_t* Xq, const int8_t* Wq, const float* t, const float* u, const uint16_t* bias,
+                         int64_t N, int64_t C1, int64_t C2, uint16_t* Yq, WorkspaceHeader* hdr, cudaStream_t st);
 
 }  // namespace tlq

@@ -216,6 +216,15 @@ __device__ __forceinline__ void scaled16(const uint4* row_smem, int64_t c, const
         v[j * 4 + 0] = __fmul_rn(src[o + 0], r.x); v[j * 4 + 1] = __fmul_rn(src[o + 1], r.y);
         v[j * 4 + 2] = __fmul_rn(src[o + 2], r.z); v[j * 4 + 3] = __fmul_rn(src[o + 3], r.w);
       }
+    } else if (s_row != nullptr) {      // single scale vector given as bf16: take the reciprocal here
+      float sa[8], sb[8];
+      unpack8(*reinterpret_cast<const uint4*>(s_row + c), sa);
+      unpack8(*reinterpret_cast<const uint4*>(s_row + c + 8), sb);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        v[j] = __fmul_rn(a[j], __fdiv_rn(1.0f, sa[j]));
+        v[8 + j] = __fmul_rn(b[j], __fdiv_rn(1.0f, sb[j]));
+      }
     } else {
 #pragma unroll
       for (int j = 0; j < 8; ++j) { v[j] = a[j]; v[8 + j] = b[j]; }
@@ -304,9 +313,9 @@ int launch_fakequant_rows_i8(const uint16_t* W, const uint16_t* s, int K, int64_
   return launch_rows<false>(W, s, nullptr, K, C2, C1, q, u, st);
 }
 
-int launch_actquant_i8(const uint16_t* X, const float* rs, int K, int64_t N, int64_t C1, int8_t* q, float* t,
-                       cudaStream_t st) {
-  return launch_rows<true>(X, nullptr, rs, K, N, C1, q, t, st);
+int launch_actquant_i8(const uint16_t* X, const uint16_t* s, const float* rs, int K, int64_t N, int64_t C1, int8_t* q,
+                       float* t, cudaStream_t st) {
+  return launch_rows<true>(X, s, rs, K, N, C1, q, t, st);
 }
 
 }  // namespace tlq

@@ -28,7 +28,7 @@ STAGE_NAMES = ("stats", "fakequant", "gemm", "reduce")
 
 EXPORTS = (
     "tlq_status_string", "tlq_version", "tlq_token_importance", "tlq_scale_candidates_workspace_bytes",
-    "tlq_scale_candidates", "tlq_quantize_weights", "tlq_scale_search_workspace_bytes", "tlq_scale_search_layer",
+    "tlq_scale_candidates", "tlq_quantize_weights", "tlq_quantize_activations", "tlq_scale_search_workspace_bytes", "tlq_scale_search_layer",
     "tlq_apply_layer_workspace_bytes", "tlq_apply_layer", "tlq_read_status", "tlq_stage_timing_enable",
     "tlq_stage_timing_drain", "tlq_kernel_launch_count",
 )
@@ -71,6 +71,8 @@ def _load() -> ctypes.CDLL:
     lib.tlq_scale_candidates_workspace_bytes.argtypes = [i64, i64]
     lib.tlq_scale_candidates.argtypes = [vp, i64, i64, vp, cfgp, vp, sz, vp, vp, vp]
     lib.tlq_quantize_weights.argtypes = [vp, vp, i64, i64, cfgp, vp, vp, vp, vp, vp]
+    lib.tlq_quantize_activations.argtypes = [vp, vp, i64, i64, cfgp, vp, vp, vp]
+    lib.tlq_quantize_activations.restype = i32
     lib.tlq_scale_search_workspace_bytes.restype = sz
     lib.tlq_scale_search_workspace_bytes.argtypes = [i64, i64, i64, cfgp]
     lib.tlq_scale_search_layer.argtypes = [vp, i64, i64, vp, i64, vp, vp, cfgp, vp, sz, vp, vp, vp, vp, vp]
@@ -80,7 +82,7 @@ def _load() -> ctypes.CDLL:
     lib.tlq_read_status.argtypes = [vp, vp]
     lib.tlq_stage_timing_enable.argtypes = [i32]
     lib.tlq_stage_timing_drain.argtypes = [ctypes.POINTER(ctypes.c_float), i32]
-    for fn in ("tlq_token_importance", "tlq_scale_candidates", "tlq_quantize_weights", "tlq_scale_search_layer",
+    for fn in ("tlq_token_importance", "tlq_scale_candidates", "tlq_quantize_weights", "tlq_quantize_activations", "tlq_scale_search_layer",
                "tlq_apply_layer", "tlq_read_status", "tlq_stage_timing_enable", "tlq_stage_timing_drain"):
         getattr(lib, fn).restype = i32
     return lib
@@ -157,6 +159,16 @@ def tlq_quantize_weights(W: torch.Tensor, s: Optional[torch.Tensor], cfg: Config
     _check(lib.tlq_quantize_weights(_ptr(W), _ptr(s), C2, C1, ctypes.byref(cfg), _ptr(codes), _ptr(steps), _ptr(zeros),
                                     _ptr(dW), _stream(stream)), "tlq_quantize_weights")
     return dict(codes=codes, steps=steps, zeros=zeros, dW=dW)
+
+
+def tlq_quantize_activations(X: torch.Tensor, s: Optional[torch.Tensor], cfg: Config, stream=None):
+    """X [N,C1] bf16, s [C1] bf16 or None -> (codes int8 [N,C1], steps float32 [N]) (W8A8 mode)."""
+    N, C1 = X.shape
+    codes = torch.empty((N, C1), dtype=torch.int8, device=X.device)
+    steps = torch.empty((N,), dtype=torch.float32, device=X.device)
+    _check(lib.tlq_quantize_activations(_ptr(X), _ptr(s), N, C1, ctypes.byref(cfg), _ptr(codes), _ptr(steps),
+                                        _stream(stream)), "tlq_quantize_activations")
+    return codes, steps
 
 
 def tlq_scale_search_workspace_bytes(N: int, C1: int, C2: int, cfg: Config) -> int:

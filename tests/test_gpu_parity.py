@@ -243,3 +243,66 @@ def test_device_errors_are_reported_not_raised_as_faults(tlq):
     assert rc == tlq.ERR_WORKSPACE
     torch.cuda.synchronize()
     assert tlq.tlq_kernel_launch_count() >= 0
+
+
+# ----------------------------------------------------------------------------------- W8A8
+
+
+@pytest.mark.parametrize("n,c1", [(64, 512), (130, 1040), (1000, 3584)])
+def test_int8_activation_quantizer_bit_exact(tlq, n, c1):
+    xb = wl.activations(11, f"a8/x{n}x{c1}", n, c1, (3 * n) // 4, "normal", 4)
+    s_np = orc.scale_table(orc.channel_stat(xb), 20)[11]
+    cfg = tlq.config(tlq.W8A8_SYM)
+    for s_vec in (None, s_np):
+        s_dev = None if s_vec is None else dev_bf16(tlq, orc.f32_to_bf16_bits(s_vec))
+        codes, steps = tlq.tlq_quantize_activations(dev_bf16(tlq, xb), s_dev, cfg)
+        torch.cuda.synchronize()
+        qx, t = orc.quantize_activations_token_sym(xb, s_vec)
+        assert np.array_equal(codes.cpu().numpy(), qx)
+        assert np.array_equal(steps.cpu().numpy().view(np.uint32), t.view(np.uint32))
+
+
+def run_search_w8a8(tlq, xb, wb, imp, n_grid=20):
+    cfg = tlq.config(tlq.W8A8_SYM, n_grid=n_grid)
+    w_dev = None if imp is None else torch.from_numpy(np.asarray(imp, dtype=np.float32)).cuda()
+    out = tlq.tlq_scale_search_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), w_dev, cfg, per_token=True)
+    return dict(best=int(out.best_idx.item()), losses=out.losses.cpu().numpy(), per_token=out.per_token.cpu().numpy(),
+                s_best=bits_of(out.s_best))
+
+
+@pytest.mark.parametrize("n,c1,c2,n_grid", [(256, 512, 512, 20), (300, 208, 320, 5), (128, 128, 256, 3), (1, 256, 64, 2),
+                                            (515, 1088, 777, 6)])
+def test_search_w8a8(tlq, n, c1, c2, n_grid):
+    xb, wb, imp = wl.small_case(43, n, c1, c2, n_outlier=2)
+    ref = orc.scale_search(xb, wb, imp, "w8a8", 0, n_grid)
+    got = run_search_w8a8(tlq, xb, wb, imp, n_grid)
+    check_against_oracle(got, ref, n_grid)
+
+
+def test_search_w8a8_importance_special_cases_and_determinism(tlq):
+    xb, wb, imp = wl.small_case(47, 384, 256, 512)
+    ref = orc.scale_search(xb, wb, None, "w8a8", 0, 6)
+    uni = run_search_w8a8(tlq, xb, wb, None, 6)
+    check_against_oracle(uni, ref, 6)
+    hot = np.zeros(384, np.float32)
+    hot[77] = 1.0
+    one = run_search_w8a8(tlq, xb, wb, hot, 6)
+    np.testing.assert_allclose(one["losses"], uni["per_token"][:, 77].astype(np.float64) / 512.0, rtol=1e-6)
+    again = run_search_w8a8(tlq, xb, wb, None, 6)
+    assert np.array_equal(uni["losses"].view(np.uint64), again["losses"].view(np.uint64))
+    assert np.array_equal(uni["per_token"].view(np.uint32), again["per_token"].view(np.uint32))
+
+
+def test_apply_layer_w8a8(tlq):
+    xb, wb, imp = wl.small_case(53, 300, 256, 328)
+    ref = orc.scale_search(xb, wb, imp, "w8a8", 0, 8)
+    s = ref["scales"][ref["best"]]
+    bias_bits = wl.f32_to_bf16_bits(np.linspace(-0.5, 0.5, 328).astype(np.float32))
+    yq_ref, (qw, u, _) = orc.apply_layer(xb, wb, s, bias_bits, "w8a8")
+    out = tlq.tlq_apply_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), dev_bf16(tlq, orc.f32_to_bf16_bits(s)),
+                              dev_bf16(tlq, bias_bits), tlq.config(tlq.W8A8_SYM))
+    assert np.array_equal(out["codes"].cpu().numpy(), qw)
+    assert np.array_equal(out["steps"].cpu().numpy().view(np.uint32), u.view(np.uint32))
+    yq = out["Yq"].float().cpu().numpy().astype(np.float64)
+    # integer accumulation is exact; what remains is the bf16 rounding of the output (2^-9 relative, doubled)
+    assert np.all(np.abs(yq - yq_ref) <= 2.0 ** -8 * np.abs(yq_ref) + 1e-6)
