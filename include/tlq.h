@@ -110,6 +110,25 @@ int tlq_scale_candidates(const void* X, int64_t N, int64_t C1, const uint8_t* ma
                          void* stream);
 
 /*
+ * tlq_scale_candidates for callers that may not allocate device memory.  (The paper has no counterpart;
+ * this is a packaging variant of the call above and computes the same x_stat and scale table.)
+ *
+ * Some hosts of this library cannot hand it a workspace: code that runs where cudaMalloc is off limits
+ * (inside a framework's allocator callback, in a process whose memory pool is fixed at start-up, in a
+ * plug-in that is only given its input and output tensors).  For them the partial sums live in a 4 MiB
+ * device array that is part of the library image, so the call needs nothing but X and the outputs.
+ *  - Limit: C1 <= 32768 (TLQ_ERR_SHAPE beyond that); N is unlimited, large N simply uses fewer, taller
+ *    row chunks than the workspace version.  Every GPU that loads the library holds the 4 MiB until exit.
+ *  - The first call on each device looks up the array's device address (with that device current) and
+ *    keeps it; make that first call outside of any stream capture.  No call allocates or frees memory.
+ *  - All calls share the one array.  Each call overwrites every partial it later reads, so nothing is
+ *    carried over from the previous call, but two calls whose kernels overlap on the GPU (different
+ *    streams, or different threads on one device) race on it: serialise them.
+ */
+int tlq_scale_candidates_noalloc(const void* X, int64_t N, int64_t C1, const uint8_t* mask, const tlq_config* cfg,
+                                 double* x_stat_out, void* s_out, void* stream);
+
+/*
  * Fake-quantize the scaled weights for ONE scale vector: Q_w(W * scale) (Sec. 3.2.1, f_q; quantizer Sec. 2.2).
  *   W [C2,C1] bf16;  s [C1] bf16 or NULL (= all ones, plain round-to-nearest)
  * Group mode: codes [C2,C1] uint8 in [0,2^w_bits-1]; steps [C2,C1/G] fp32; zeros [C2,C1/G] int32;

@@ -198,6 +198,22 @@ int tlq_scale_candidates(const void* X, int64_t N, int64_t C1, const uint8_t* ma
                             reinterpret_cast<uint16_t*>(s_out), nullptr, st);
 }
 
+int tlq_scale_candidates_noalloc(const void* X, int64_t N, int64_t C1, const uint8_t* mask, const tlq_config* cfg,
+                                 double* x_stat_out, void* s_out, void* stream) {
+  if (X == nullptr || s_out == nullptr) return TLQ_ERR_INVALID_ARG;
+  if (N < 1) return TLQ_ERR_SHAPE;
+  int rc = check_cfg(cfg, C1, false);
+  if (rc != TLQ_OK) return rc;
+  if (C1 > static_stats_max_c1()) return TLQ_ERR_SHAPE;   // beyond the built-in scratch
+  if (cfg->stat_mode == TLQ_STAT_MASKED_MAX && mask == nullptr) return TLQ_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(s_out)) return TLQ_ERR_ALIGN;
+  rc = have_device();
+  if (rc != TLQ_OK) return rc;
+  return launch_scale_candidates_static(reinterpret_cast<const uint16_t*>(X), N, C1, mask, cfg->stat_mode, cfg->n_grid,
+                                        x_stat_out, reinterpret_cast<uint16_t*>(s_out),
+                                        reinterpret_cast<cudaStream_t>(stream));
+}
+
 int tlq_quantize_weights(const void* W, const void* s, int64_t C2, int64_t C1, const tlq_config* cfg, uint8_t* codes,
                          float* steps, int32_t* zeros, void* dW_out, void* stream) {
   if (W == nullptr) return TLQ_ERR_INVALID_ARG;

@@ -82,6 +82,10 @@ int launch_scale_table(const double* partials, int64_t chunks, int64_t N, int64_
                        double* x_stat /*[C1] or null*/, uint16_t* s /*[K,C1]*/, float* rs /*[K,C1] or null*/,
                        cudaStream_t st);
 
+int64_t static_stats_max_c1();
+int launch_scale_candidates_static(const uint16_t* X, int64_t N, int64_t C1, const uint8_t* mask, int stat_mode, int K,
+                                   double* x_stat /*[C1] or null*/, uint16_t* s /*[K,C1]*/, cudaStream_t st);
+
 // fakequant.cu
 int launch_fakequant_group(const uint16_t* W, const uint16_t* s /*[K,C1] or null*/, const float* rs /*[K,C1] or null: 1/s*/,
                            int K, int64_t C2, int64_t C1,

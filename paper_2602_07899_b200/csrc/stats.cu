@@ -120,4 +120,64 @@ int launch_scale_table(const double* partials, int64_t chunks, int64_t N, int64_
   return after_launch();
 }
 
+// ------------------------------------------------------------------------------------------------
+// Variant for callers that cannot allocate device memory: the per-chunk column partials live in a
+// file-scope device array instead of a caller-provided workspace.  The array belongs to the loaded
+// library image: every GPU that loads the library holds these 4 MiB until the process exits.
+// ------------------------------------------------------------------------------------------------
+constexpr int64_t kStaticScratchDoubles = 524288;     // 4 MiB of fp64 partials
+constexpr int64_t kStaticMaxC1 = 32768;               // leaves room for at least 16 row chunks
+static __device__ __align__(256) double g_static_partials[kStaticScratchDoubles];
+
+int64_t static_stats_max_c1() { return kStaticMaxC1; }
+
+// In host code `g_static_partials` is only a handle for the symbol, not a device address; the address a
+// kernel can use is looked up once per device (with that device current) and cached here.
+static double* static_partials_ptr(int* status) {
+  constexpr int kMaxDevices = 64;
+  static double* cached[kMaxDevices] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { *status = TLQ_ERR_CUDA; return nullptr; }
+  if (cached[dev] == nullptr) {
+    double* p = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_partials) != cudaSuccess || p == nullptr) {
+      cudaGetLastError();
+      *status = TLQ_ERR_CUDA;
+      return nullptr;
+    }
+    cached[dev] = p;
+  }
+  *status = TLQ_OK;
+  return cached[dev];
+}
+
+int launch_scale_candidates_static(const uint16_t* X, int64_t N, int64_t C1, const uint8_t* mask, int stat_mode, int K,
+                                   double* x_stat, uint16_t* s, cudaStream_t st) {
+  int rc = TLQ_OK;
+  double* partials = static_partials_ptr(&rc);
+  if (rc != TLQ_OK) return rc;
+  // as many row chunks as the regular path would use, capped by what the fixed array can hold
+  int64_t chunks = stats_row_chunks(N);
+  const int64_t cap = kStaticScratchDoubles / C1;
+  if (chunks > cap) chunks = cap;
+  const int64_t rows_per_chunk = ceil_div(N, chunks);
+  chunks = ceil_div(N, rows_per_chunk);
+  dim3 grid((unsigned)ceil_div(C1, kStatTx * 8), (unsigned)chunks), block(kStatTx, kStatTy);
+  // every partial in [0, chunks) x [0, C1) is overwritten before the second stage reads it, so nothing
+  // left behind by an earlier call can reach the result and nothing needs clearing
+  switch (stat_mode) {
+    case TLQ_STAT_MEAN_ABS:
+      channel_stats_kernel<TLQ_STAT_MEAN_ABS><<<grid, block, 0, st>>>(X, N, C1, mask, rows_per_chunk, partials);
+      break;
+    case TLQ_STAT_MAX_ABS:
+      channel_stats_kernel<TLQ_STAT_MAX_ABS><<<grid, block, 0, st>>>(X, N, C1, mask, rows_per_chunk, partials);
+      break;
+    default:
+      channel_stats_kernel<TLQ_STAT_MASKED_MAX><<<grid, block, 0, st>>>(X, N, C1, mask, rows_per_chunk, partials);
+      break;
+  }
+  if ((rc = after_launch()) != TLQ_OK) return rc;
+  return launch_scale_table(partials, chunks, N, C1, stat_mode, K, x_stat, s, nullptr, st);
+}
+
 }  // namespace tlq

@@ -28,7 +28,7 @@ STAGE_NAMES = ("stats", "fakequant", "gemm", "reduce")
 
 EXPORTS = (
     "tlq_status_string", "tlq_version", "tlq_token_importance", "tlq_scale_candidates_workspace_bytes",
-    "tlq_scale_candidates", "tlq_quantize_weights", "tlq_quantize_activations", "tlq_scale_search_workspace_bytes", "tlq_scale_search_layer",
+    "tlq_scale_candidates", "tlq_scale_candidates_noalloc", "tlq_quantize_weights", "tlq_quantize_activations", "tlq_scale_search_workspace_bytes", "tlq_scale_search_layer",
     "tlq_apply_layer_workspace_bytes", "tlq_apply_layer", "tlq_read_status", "tlq_stage_timing_enable",
     "tlq_stage_timing_drain", "tlq_kernel_launch_count",
 )
@@ -70,6 +70,8 @@ def _load() -> ctypes.CDLL:
     lib.tlq_scale_candidates_workspace_bytes.restype = sz
     lib.tlq_scale_candidates_workspace_bytes.argtypes = [i64, i64]
     lib.tlq_scale_candidates.argtypes = [vp, i64, i64, vp, cfgp, vp, sz, vp, vp, vp]
+    lib.tlq_scale_candidates_noalloc.argtypes = [vp, i64, i64, vp, cfgp, vp, vp, vp]
+    lib.tlq_scale_candidates_noalloc.restype = i32
     lib.tlq_quantize_weights.argtypes = [vp, vp, i64, i64, cfgp, vp, vp, vp, vp, vp]
     lib.tlq_quantize_activations.argtypes = [vp, vp, i64, i64, cfgp, vp, vp, vp]
     lib.tlq_quantize_activations.restype = i32
@@ -82,7 +84,7 @@ def _load() -> ctypes.CDLL:
     lib.tlq_read_status.argtypes = [vp, vp]
     lib.tlq_stage_timing_enable.argtypes = [i32]
     lib.tlq_stage_timing_drain.argtypes = [ctypes.POINTER(ctypes.c_float), i32]
-    for fn in ("tlq_token_importance", "tlq_scale_candidates", "tlq_quantize_weights", "tlq_quantize_activations", "tlq_scale_search_layer",
+    for fn in ("tlq_token_importance", "tlq_scale_candidates", "tlq_scale_candidates_noalloc", "tlq_quantize_weights", "tlq_quantize_activations", "tlq_scale_search_layer",
                "tlq_apply_layer", "tlq_read_status", "tlq_stage_timing_enable", "tlq_stage_timing_drain"):
         getattr(lib, fn).restype = i32
     return lib
@@ -140,6 +142,15 @@ def tlq_scale_candidates(X: torch.Tensor, cfg: Config, mask: Optional[torch.Tens
     _check(lib.tlq_scale_candidates(_ptr(X), N, C1, _ptr(mask), ctypes.byref(cfg), _ptr(ws), nbytes, _ptr(x_stat),
                                     _ptr(s), _stream(stream)), "tlq_scale_candidates")
     return x_stat, s
+
+
+def tlq_scale_candidates_noalloc(X: torch.Tensor, cfg: Config, x_stat: torch.Tensor, s: torch.Tensor,
+                                 mask: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Same result as tlq_scale_candidates, written into the caller's x_stat [C1] float64 and s [K,C1] bf16;
+    the library uses its built-in scratch array, so nothing is allocated here or in the library."""
+    N, C1 = X.shape
+    _check(lib.tlq_scale_candidates_noalloc(_ptr(X), N, C1, _ptr(mask), ctypes.byref(cfg), _ptr(x_stat), _ptr(s),
+                                            _stream(stream)), "tlq_scale_candidates_noalloc")
 
 
 def tlq_quantize_weights(W: torch.Tensor, s: Optional[torch.Tensor], cfg: Config, want_dw: bool = False, stream=None):
