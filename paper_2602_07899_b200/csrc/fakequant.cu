@@ -5,7 +5,7 @@
 // in shared memory and re-used for every scale candidate, so the source is read once and each
 // candidate's operand is written once.  The arithmetic is kept off the slow conversion / reciprocal
 // unit: rounding to an integer is the add-and-subtract of 1.5*2^23 (exact round-half-even in
-// binary32 for |x| < 2^22), clamping stays in floating point, int8 codes are read out of the low
+// binary32 for |x| < 2^22), clamping is done before rounding and in floating point, int8 codes are read out of the low
 // mantissa bits, and the per-element quotient value/step is taken as value * (1/step) with an exact
 // IEEE division only when the product lies so close to a rounding tie that the two could round
 // differently.  The integer produced is therefore always rint(fl32(value / step)), the contract the
@@ -21,19 +21,29 @@ constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23
 // rint(x) for |x| <= 2^21 without a conversion instruction.
 __device__ __forceinline__ float round_magic(float x) { return __fsub_rn(__fadd_rn(x, kMagic), kMagic); }
 
-// rint(fl32(v / step)) given inv = fl32(1 / step).
-// fl32(v * inv) is within |q| * 1.8e-7 of the true quotient and so is fl32(v / step); for |q| < 1024
-// that is below 2.5e-4, so when the product is farther than that from a tie both round to the same
-// integer.  For |q| >= 1024 every caller clamps to a range inside (-1024, 1024), where the integer
-// is saturated whichever way the quotient rounds.
-__device__ __forceinline__ float quotient_rint(float v, float step, float inv) {
-  float q = __fmul_rn(v, inv);
-  q = fminf(fmaxf(q, -2097152.0f), 2097152.0f);
+// Reciprocal to within one ulp (a single instruction on the special-function unit).
+__device__ __forceinline__ float rcp_fast(float x) {
+  float r;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r;
+}
+
+// The rare exact path, kept out of line so the common path stays a dozen instructions.
+__device__ __noinline__ float exact_quotient_rint(float v, float step, float lo, float hi) {
+  const float exact = fminf(fmaxf(__fdiv_rn(v, step), lo), hi);
+  return round_magic(exact);
+}
+
+// clamp(rint(fl32(v / step)), lo, hi) for integer bounds lo <= hi inside (-1024, 1024), given
+// inv ~ 1/step to within one ulp.  Clamping before rounding gives the same integer because the bounds
+// are integers and rounding is monotone.  fl32(v * inv) is within |q| * 2.4e-7 of the true quotient
+// and fl32(v / step) within |q| * 6e-8, so with |q| < 1024 both lie within 2.5e-4 of it: when the
+// product is farther than that from a rounding tie the two round to the same integer, otherwise the
+// exact division decides.
+__device__ __forceinline__ float quotient_rint_clamped(float v, float step, float inv, float lo, float hi) {
+  const float q = fminf(fmaxf(__fmul_rn(v, inv), lo), hi);
   float r = round_magic(q);
-  if (fabsf(__fsub_rn(q, r)) > 0.49975f && fabsf(q) < 1024.0f) {
-    const float exact = __fdiv_rn(v, step);
-    r = round_magic(exact);
-  }
+  if (fabsf(__fsub_rn(q, r)) > 0.49975f) r = exact_quotient_rint(v, step, lo, hi);
   return r;
 }
 
@@ -136,10 +146,10 @@ fakequant_group_kernel(const uint16_t* __restrict__ W, const uint16_t* __restric
       }
       const float range = fmaxf(__fsub_rn(mx, mn), TLQ_RANGE_FLOOR);
       const float step = __fdiv_rn(range, qmax_f);
-      const float inv = __fdiv_rn(1.0f, step);
-      int z = -__float2int_rn(__fdiv_rn(mn, step));
-      z = min(max(z, 0), qmax);
-      const float zf = (float)z;
+      const float inv = rcp_fast(step);
+      // zero-point z = clamp(-rint(mn / step), 0, qmax), kept as a float
+      const float zf = -quotient_rint_clamped(mn, step, inv, -qmax_f, 0.0f);
+      const float lo = -zf, hi = qmax_f - zf;          // bounds of q - z
       uint32_t outw[8];
       uint32_t qpack[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
@@ -147,13 +157,12 @@ fakequant_group_kernel(const uint16_t* __restrict__ W, const uint16_t* __restric
         float d[2];
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-          float q = __fadd_rn(quotient_rint(pr[j + h], step, inv), zf);
-          q = fminf(fmaxf(q, 0.0f), qmax_f);
-          const float dq = __fmul_rn(__fsub_rn(q, zf), step);
+          const float qz = quotient_rint_clamped(pr[j + h], step, inv, lo, hi);     // q - z
+          const float dq = __fmul_rn(qz, step);
           const float w_hat = __fmul_rn(dq, rsv[j + h]);
           d[h] = __fsub_rn(w[j + h], w_hat);
           if (codes != nullptr)
-            qpack[(j + h) >> 2] |= (__float_as_uint(__fadd_rn(q, kMagic)) & 0xFFu) << (((j + h) & 3) * 8);
+            qpack[(j + h) >> 2] |= (__float_as_uint(__fadd_rn(__fadd_rn(qz, zf), kMagic)) & 0xFFu) << (((j + h) & 3) * 8);
         }
         outw[j >> 1] = pack_bf16x2(d[0], d[1]);
       }
@@ -169,7 +178,7 @@ fakequant_group_kernel(const uint16_t* __restrict__ W, const uint16_t* __restric
         if ((lane % lanes_per_group) == 0) {
           const int64_t g = c0 / group;
           if (steps != nullptr) steps[row * ngroups + g] = step;
-          if (zeros != nullptr) zeros[row * ngroups + g] = z;
+          if (zeros != nullptr) zeros[row * ngroups + g] = (int)zf;
         }
       }
     }
@@ -274,7 +283,7 @@ quant_rows_i8_kernel(const uint16_t* __restrict__ src, const uint16_t* __restric
 #pragma unroll
       for (int w = 1; w < kRowThreads / 32; ++w) m = fmaxf(m, wm[w]);
       const float st = __fdiv_rn(fmaxf(m, TLQ_RANGE_FLOOR), 127.0f);
-      const float inv = __fdiv_rn(1.0f, st);
+      const float inv = rcp_fast(st);
       if (t == 0) step_out[(int64_t)k * R + row] = st;
       int8_t* out = q + ((int64_t)k * R + row) * C1;
       for (int64_t c = (int64_t)t * 16; c < C1; c += kRowThreads * 16) {
@@ -283,8 +292,7 @@ quant_rows_i8_kernel(const uint16_t* __restrict__ src, const uint16_t* __restric
         uint32_t pk[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-          float qi = quotient_rint(v[j], st, inv);
-          qi = fminf(fmaxf(qi, -128.0f), 127.0f);
+          const float qi = quotient_rint_clamped(v[j], st, inv, -128.0f, 127.0f);
           pk[j >> 2] |= (__float_as_uint(__fadd_rn(qi, kMagic)) & 0xFFu) << ((j & 3) * 8);
         }
         *reinterpret_cast<uint4*>(out + c) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
