@@ -30,7 +30,8 @@ import numpy as np  # noqa: E402
 METRIC = "scale_grid_candidates_per_sec"
 UNIT = "candidates/s"
 SAMPLE_LINEAR = "k"
-SAMPLE_TOKENS = 2048
+SAMPLE_TOKENS = 2048           # per step of the reference arm (many steps: keep each near a second)
+BASELINE_TOKENS = 16384        # the one-shot cpu_baseline leg of the GPU arm (about 5-20 s of CPU work)
 
 
 def measured_peaks():
@@ -50,12 +51,12 @@ def layer_flops(cfgw):
 # --------------------------------------------------------------------------------------------- CPU oracle legs
 
 
-def oracle_sample_seconds(cfgw, data):
-    """One pass of the oracle over the bounded sample: one projection, the first SAMPLE_TOKENS tokens,
+def oracle_sample_seconds(cfgw, data, tokens=SAMPLE_TOKENS):
+    """One pass of the oracle over the bounded sample: one projection, the first `tokens` tokens,
     all K candidates.  Returns (seconds, flops of the sample)."""
     from oracle import tlq_oracle as orc
     lin = cfgw.linear(SAMPLE_LINEAR)
-    n = min(SAMPLE_TOKENS, cfgw.n_tokens)
+    n = min(tokens, cfgw.n_tokens)
     x, w, imp = data.x(lin)[:n], data.w(lin), data.imp()[:n]
     t0 = time.perf_counter()
     orc.scale_search(x, w, imp, cfgw.mode, cfgw.group, cfgw.n_grid)
@@ -63,9 +64,9 @@ def oracle_sample_seconds(cfgw, data):
     return dt, 2.0 * n * lin.c_in * lin.c_out * cfgw.n_grid
 
 
-def sample_description(cfgw):
+def sample_description(cfgw, tokens=SAMPLE_TOKENS):
     lin = cfgw.linear(SAMPLE_LINEAR)
-    n = min(SAMPLE_TOKENS, cfgw.n_tokens)
+    n = min(tokens, cfgw.n_tokens)
     return (f"{SAMPLE_LINEAR}-projection {lin.c_in}->{lin.c_out}, first {n} of {cfgw.n_tokens} tokens, all "
             f"{cfgw.n_grid} candidates; scaled to the whole layer by 2*N*C1*C2*K (extrapolated)")
 
@@ -76,10 +77,9 @@ def candidates_per_sec_from_sample(cfgw, seconds, flops):
 
 
 def run_reference(args, cfgw):
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
-        return
-    from paper_2602_07899_b200 import workloads as wl
+    from paper_2602_07899_b200 import replicas, workloads as wl
+    if not replicas.rank_info_from_env().is_root:
+        return      # rank 0 alone runs and prints the reference arm
     data = wl.LayerData(cfgw)
     for _ in range(args.warmup):
         oracle_sample_seconds(cfgw, data)
@@ -162,16 +162,14 @@ def run_ours(args, cfgw):
     import torch.distributed as dist
     from paper_2602_07899_b200 import tlq, workloads as wl
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2602_07899_b200 import replicas
+    info = replicas.rank_info_from_env()
+    world, rank, local = info.world, info.rank, info.local_rank
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=dev)
+    replicas.init_process_group(info, "nccl", dev)
 
     def barrier():
         if world > 1:
@@ -180,7 +178,7 @@ def run_ours(args, cfgw):
 
     # every rank calibrates its own layer: same shapes, its own seed
     import dataclasses
-    cfgr = dataclasses.replace(cfgw, seed=cfgw.seed + rank)
+    cfgr = dataclasses.replace(cfgw, seed=replicas.replica_seed(cfgw.seed, rank))
     data = wl.LayerData(cfgr)
     lins = [l for l in cfgr.linears() if args.linears is None or l.name in args.linears.split(",")]
     mode = tlq.W4A16_ASYM_GROUP if cfgr.mode == "w4a16" else tlq.W8A8_SYM
@@ -270,14 +268,11 @@ def run_ours(args, cfgw):
     assert all(int(out_host[l.name][0].item()) == best[l.name] for l in lins)
 
     # ---- max over ranks
-    if world > 1:
-        t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, ms_e2e = float(t[0]), float(t[1])
+    ms_total, ms_e2e = replicas.max_over_ranks([ms_total, ms_e2e], info, dev)
 
     n_cand_step = len(lins) * cfgr.n_grid
-    value = world * n_cand_step * args.steps / (ms_total * 1e-3)
-    e2e_value = world * n_cand_step * args.steps / (ms_e2e * 1e-3)
+    value = replicas.whole_job_rate(n_cand_step, args.steps, info, ms_total)
+    e2e_value = replicas.whole_job_rate(n_cand_step, args.steps, info, ms_e2e)
 
     # ---- roofline of the dominant kernel (the fused search GEMM), from the per-stage events of the timed region
     peaks = measured_peaks()
@@ -298,7 +293,18 @@ def run_ours(args, cfgw):
     lin_report = {}
     for name, d in per_linear.items():
         g = statistics.mean(d["gemm_ms"])
+        l = next(x for x in lins if x.name == name)
+        K = cfgr.n_grid
+        # algorithmic bytes of the two streaming stages: X read once (+ the two K x C1 scale tables);
+        # W read once and K operands written (bf16 delta weights, or int8 weights + int8 activations)
+        stat_bytes = 2.0 * cfgr.n_tokens * l.c_in + 6.0 * K * l.c_in
+        if cfgr.mode == "w4a16":
+            fq_bytes = (2.0 + 2.0 * K) * l.c_out * l.c_in
+        else:
+            fq_bytes = (2.0 + K) * l.c_out * l.c_in + (2.0 + K) * cfgr.n_tokens * l.c_in
         lin_report[name] = {"gemm_ms": round(g, 4), "gemm_tflops": round(d["flops"] / (g * 1e-3) / 1e12, 1),
+                            "stats_gbs": round(stat_bytes / (d["stages_ms"][0] / n_rec * 1e-3) / 1e9, 1),
+                            "fakequant_gbs": round(fq_bytes / (d["stages_ms"][1] / n_rec * 1e-3) / 1e9, 1),
                             "stages_ms": [round(v / n_rec, 4) for v in d["stages_ms"]],
                             "candidates_per_s": round(cfgr.n_grid / (sum(d["stages_ms"]) / n_rec * 1e-3), 1),
                             "best_idx": best[name]}
@@ -308,11 +314,18 @@ def run_ours(args, cfgw):
     if os.path.exists(tpath):
         with open(tpath) as f:
             traffic = json.load(f).get(cfgr.key)
-    roofline = {"kernel": "gemm_bf16_kernel<search>", "bound": "tensor", "achieved": achieved,
-                "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
-                "frac": (achieved / peaks["bf16_sustained"]) if achieved else None, "traffic": traffic,
-                "peak_source": f"{peaks['source']} (sustained cuBLAS bf16; burst {peaks['bf16_burst']})",
-                "frac_of_nominal_2250": (achieved / 2250.0) if achieved else None,
+    i8 = cfgr.mode != "w4a16"
+    # int8 runs at twice the bf16 rate on these tensor cores (nominal 4500 vs 2250 dense): the int8 peak
+    # is the measured bf16 peak times that nominal ratio
+    ratio = 2.0 if i8 else 1.0
+    peak = peaks["bf16_sustained"] * ratio
+    nominal = 2250.0 * ratio
+    roofline = {"kernel": "gemm_w8a8_kernel<search>" if i8 else "gemm_bf16_kernel<search>", "bound": "tensor",
+                "achieved": achieved, "peak": peak, "unit": "TOP/s" if i8 else "TFLOP/s",
+                "frac": (achieved / peak) if achieved else None, "traffic": traffic,
+                "peak_source": (f"{peaks['source']} (sustained cuBLAS bf16 {peaks['bf16_sustained']}"
+                                f"{' x2 nominal int8:bf16 ratio' if i8 else ''}; burst {peaks['bf16_burst']})"),
+                "frac_of_nominal": (achieved / nominal) if achieved else None, "nominal_peak": nominal,
                 "launches_timed": len(stage_ms),
                 "stage_share": {n: round(v / max(sum(stage_tot), 1e-9), 4) for n, v in zip(tlq.STAGE_NAMES, stage_tot)}}
 
@@ -323,9 +336,9 @@ def run_ours(args, cfgw):
 
     cpu = None
     if world == 1:
-        dt, fl = oracle_sample_seconds(cfgw, data)
+        dt, fl = oracle_sample_seconds(cfgw, data, BASELINE_TOKENS)
         cpu = {"value": candidates_per_sec_from_sample(cfgw, dt, fl), "unit": UNIT, "cores": os.cpu_count(),
-               "kind": "oracle", "sample": sample_description(cfgw), "sample_seconds": round(dt, 3),
+               "kind": "oracle", "sample": sample_description(cfgw, BASELINE_TOKENS), "sample_seconds": round(dt, 3),
                "oracle_gflops": round(fl / dt / 1e9, 1)}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -345,7 +358,7 @@ def run_ours(args, cfgw):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="cfg1")
