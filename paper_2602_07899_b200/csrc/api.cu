@@ -232,7 +232,7 @@ int tlq_quantize_weights(const void* W, const void* s, int64_t C2, int64_t C1, c
     return launch_fakequant_group(Wb, sb, nullptr, 1, C2, C1, cfg->group_size, cfg->w_bits, reinterpret_cast<uint16_t*>(dW_out),
                                   codes, steps, zeros, st);
   if (dW_out != nullptr || codes == nullptr || steps == nullptr) return TLQ_ERR_INVALID_ARG;
-  return launch_fakequant_rows_i8(Wb, sb, 1, C2, C1, reinterpret_cast<int8_t*>(codes), steps, st);
+  return launch_fakequant_rows_i8(Wb, sb, 1, C2, C1, cfg->w_bits, reinterpret_cast<int8_t*>(codes), steps, st);
 }
 
 int tlq_quantize_activations(const void* X, const void* s, int64_t N, int64_t C1, const tlq_config* cfg, int8_t* codes,
@@ -246,7 +246,7 @@ int tlq_quantize_activations(const void* X, const void* s, int64_t N, int64_t C1
   rc = have_device();
   if (rc != TLQ_OK) return rc;
   return launch_actquant_i8(reinterpret_cast<const uint16_t*>(X), reinterpret_cast<const uint16_t*>(s), nullptr, 1, N,
-                            C1, codes, steps, reinterpret_cast<cudaStream_t>(stream));
+                            C1, cfg->a_bits, codes, steps, reinterpret_cast<cudaStream_t>(stream));
 }
 
 size_t tlq_scale_search_workspace_bytes(int64_t N, int64_t C1, int64_t C2, const tlq_config* cfg) {
@@ -288,8 +288,8 @@ int tlq_scale_search_layer(const void* X, int64_t N, int64_t C1, const void* W, 
     if ((rc = timing_mark(2, st)) != TLQ_OK) return rc;
     if ((rc = launch_search_gemm_bf16(Xb, L.dW, w_imp, L.plan, L.partials, ptab, L.hdr, st)) != TLQ_OK) return rc;
   } else {
-    if ((rc = launch_fakequant_rows_i8(Wb, L.s, K, C2, C1, L.Wq, L.u, st)) != TLQ_OK) return rc;
-    if ((rc = launch_actquant_i8(Xb, nullptr, L.rs, K, N, C1, L.Xq, L.t, st)) != TLQ_OK) return rc;
+    if ((rc = launch_fakequant_rows_i8(Wb, L.s, K, C2, C1, cfg->w_bits, L.Wq, L.u, st)) != TLQ_OK) return rc;
+    if ((rc = launch_actquant_i8(Xb, nullptr, L.rs, K, N, C1, cfg->a_bits, L.Xq, L.t, st)) != TLQ_OK) return rc;
     if ((rc = timing_mark(2, st)) != TLQ_OK) return rc;
     if ((rc = launch_search_gemm_i8(Xb, Wb, L.Xq, L.Wq, L.t, L.u, w_imp, L.plan, L.partials, ptab, L.hdr, st)) !=
         TLQ_OK)
@@ -363,8 +363,8 @@ int tlq_apply_layer(const void* X, int64_t N, int64_t C1, const void* W, int64_t
       return rc;
     return launch_apply_gemm_bf16(Xb, Wb, L.dW, bb, N, C1, C2, reinterpret_cast<uint16_t*>(Yq), L.hdr, st);
   }
-  if ((rc = launch_fakequant_rows_i8(Wb, sb, 1, C2, C1, L.Wq, L.u, st)) != TLQ_OK) return rc;
-  if ((rc = launch_actquant_i8(Xb, sb, nullptr, 1, N, C1, L.Xq, L.t, st)) != TLQ_OK) return rc;
+  if ((rc = launch_fakequant_rows_i8(Wb, sb, 1, C2, C1, cfg->w_bits, L.Wq, L.u, st)) != TLQ_OK) return rc;
+  if ((rc = launch_actquant_i8(Xb, sb, nullptr, 1, N, C1, cfg->a_bits, L.Xq, L.t, st)) != TLQ_OK) return rc;
   if (codes != nullptr) TLQ_CUDA_TRY(cudaMemcpyAsync(codes, L.Wq, (size_t)C2 * C1, cudaMemcpyDeviceToDevice, st));
   if (steps != nullptr) TLQ_CUDA_TRY(cudaMemcpyAsync(steps, L.u, (size_t)C2 * sizeof(float), cudaMemcpyDeviceToDevice, st));
   return launch_apply_gemm_i8(L.Xq, L.Wq, L.t, L.u, bb, N, C1, C2, reinterpret_cast<uint16_t*>(Yq), L.hdr, st);

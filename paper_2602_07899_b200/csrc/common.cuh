@@ -60,6 +60,44 @@ __device__ __forceinline__ uint4 ld_nc_16(const void* p) {
 }
 
 // ---------------------------------------------------------------------------------------------
+// Walk order of the (token tile, output tile) grid of one GEMM.  The persistent CTAs take tiles
+// round-robin from one linear order, so the tiles in flight at any moment are a run of consecutive
+// indices.  With a = mtiles the order is "all token tiles of one output tile, then the next output
+// tile": a run touches every activation tile and two or three weight tiles, which reads the weights
+// from HBM once as long as the activations stay in L2.  When they cannot (the wide down-projection),
+// a run is made a block of `a` token tiles x `b` output tiles instead, blocks advancing along the
+// tokens first: the run then needs a activation tiles and b weight tiles, and measured HBM traffic
+// of the 18944-channel case drops by a quarter.  (Measured the other way round for activations that do
+// fit, where the blocked walk re-reads weight tiles: hence the switch.)
+// ---------------------------------------------------------------------------------------------
+struct TileRaster {
+  int mtiles, otiles, a, b;
+  __host__ __device__ void decode(int64_t t, int& mt, int& ot) const {
+    const int64_t band_tiles = (int64_t)mtiles * b;
+    const int oband = (int)(t / band_tiles);
+    const int b_eff = (otiles - oband * b) < b ? (otiles - oband * b) : b;
+    int64_t r = t - (int64_t)oband * band_tiles;
+    const int mgroup = (int)(r / ((int64_t)a * b_eff));
+    const int a_eff = (mtiles - mgroup * a) < a ? (mtiles - mgroup * a) : a;
+    r -= (int64_t)mgroup * a * b_eff;
+    ot = oband * b + (int)(r / a_eff);
+    mt = mgroup * a + (int)(r % a_eff);
+  }
+};
+// `act_bytes`: bytes of the activation operand one candidate streams (bf16 X, or one candidate's int8 codes).
+inline TileRaster make_raster(int64_t mtiles, int64_t otiles, int grid, int64_t act_bytes) {
+  TileRaster r;
+  r.mtiles = (int)mtiles; r.otiles = (int)otiles;
+  if (act_bytes <= (64ll << 20)) {      // fits in half of L2 with room for the weight stream
+    r.a = (int)mtiles; r.b = 1;
+  } else {                              // 16 x grid/16 balances the bytes of 128-row and 256-row tiles
+    r.a = 16;
+    r.b = grid / 16 > 0 ? grid / 16 : 1;
+  }
+  return r;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Workspace header (first 256 bytes of every workspace)
 // ---------------------------------------------------------------------------------------------
 struct WorkspaceHeader {
@@ -91,10 +129,11 @@ int launch_fakequant_group(const uint16_t* W, const uint16_t* s /*[K,C1] or null
                            int K, int64_t C2, int64_t C1,
                            int group, int w_bits, uint16_t* dW /*[K,C2,C1] or null*/, uint8_t* codes, float* steps,
                            int32_t* zeros, cudaStream_t st);
+// symmetric `bits`-wide codes (2..8) in int8 containers
 int launch_fakequant_rows_i8(const uint16_t* W, const uint16_t* s /*[K,C1] or null*/, int K, int64_t C2, int64_t C1,
-                             int8_t* q /*[K,C2,C1]*/, float* u /*[K,C2]*/, cudaStream_t st);
+                             int bits, int8_t* q /*[K,C2,C1]*/, float* u /*[K,C2]*/, cudaStream_t st);
 // activations: x * (1/s); give the reciprocal table rs [K,C1], or a bf16 scale s [K,C1] to invert on the fly, or neither
-int launch_actquant_i8(const uint16_t* X, const uint16_t* s, const float* rs, int K, int64_t N, int64_t C1,
+int launch_actquant_i8(const uint16_t* X, const uint16_t* s, const float* rs, int K, int64_t N, int64_t C1, int bits,
                        int8_t* q /*[K,N,C1]*/, float* t /*[K,N]*/, cudaStream_t st);
 
 // importance.cu

@@ -47,6 +47,43 @@ __device__ __forceinline__ float quotient_rint_clamped(float v, float step, floa
   return r;
 }
 
+// ---- packed binary32 pairs: one instruction carries two independent IEEE round-to-nearest operations
+__device__ __forceinline__ float2 mul2(float2 a, float2 b) {
+  float2 r;
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+      "mul.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(r.x), "=f"(r.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+  return r;
+}
+__device__ __forceinline__ float2 add2(float2 a, float2 b) {
+  float2 r;
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+      "add.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(r.x), "=f"(r.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+  return r;
+}
+__device__ __forceinline__ float2 sub2(float2 a, float2 b) {
+  float2 r;
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+      "sub.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(r.x), "=f"(r.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+  return r;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+__device__ __forceinline__ float min3(float a, float b, float c) {
+  float r;
+  asm("min.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+// two bf16 values packed in a 32-bit word -> their binary32 values (low half first)
+__device__ __forceinline__ float2 unpack2(uint32_t v) {
+  return make_float2(__uint_as_float(v << 16), __uint_as_float(v & 0xFFFF0000u));
+}
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
@@ -65,6 +102,174 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 constexpr int kGqRows = 32;
 constexpr int kGqCols = 512;
 constexpr int kGqThreads = 256;
+
+// ------------------------------------------------------------------------------------------------
+// The search's own fake-quant pass: delta weights of ALL candidates, nothing else.  Same tile and
+// thread mapping as the general kernel below, but the inner loop is straight-line code on packed
+// binary32 pairs with no clamps and no per-element branch:
+//   * a group whose extreme quotients mn/step and mx/step round to integers ra <= 0 <= rb with
+//     -ra <= qmax and rb - ra <= qmax cannot clip: every element's quotient lies between the two
+//     (division and rounding are monotone), so code = rint(p/step) - ra is already inside [0, qmax]
+//     and q - z is just rint(p/step);
+//   * rint(p * (1/step)) equals rint(fl32(p/step)) unless the product lies within `tie_eps` of a
+//     rounding tie; the distance to the nearest integer is folded into one running maximum per
+//     thread and checked once per 16 elements.
+// A group that can clip, and a thread that met a near-tie, redo their 16 elements on the general
+// path (clamps, exact division), which computes the contract literally.  Both cases are rare.
+// ------------------------------------------------------------------------------------------------
+// One thread's 16 elements on the literal path (clamps, exact division near ties): the group's step,
+// its reciprocal and its minimum are given, the rest is re-read from the staged tile and the tables.
+__device__ __noinline__ void delta16_general(const uint4* tile16, const uint16_t* s16, const float* rs16, float mn,
+                                             float step, float inv, float qmax_f, uint4* dst) {
+  const float zf = -quotient_rint_clamped(mn, step, inv, -qmax_f, 0.0f);
+  const float lo = -zf, hi = qmax_f - zf;
+#pragma unroll 1
+  for (int h = 0; h < 2; ++h) {
+    float w[8], sv[8];
+    unpack8(tile16[h], w);
+    unpack8(*reinterpret_cast<const uint4*>(s16 + h * 8), sv);
+    uint32_t o[4];
+#pragma unroll
+    for (int j = 0; j < 8; j += 2) {
+      float d[2];
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const float qz = quotient_rint_clamped(__fmul_rn(sv[j + e], w[j + e]), step, inv, lo, hi);
+        d[e] = __fsub_rn(w[j + e], __fmul_rn(__fmul_rn(qz, step), rs16[h * 8 + j + e]));
+      }
+      o[j >> 1] = pack_bf16x2(d[0], d[1]);
+    }
+    dst[h] = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+
+__global__ void __launch_bounds__(kGqThreads, 2)
+fakequant_delta_kernel(const uint16_t* __restrict__ W, const uint16_t* __restrict__ s_tab,
+                       const float* __restrict__ rs_tab, int K, int k_per_cta, int64_t C2, int64_t C1, int group,
+                       int qmax, float tie_eps, uint16_t* __restrict__ dW) {
+  __shared__ uint4 tile[kGqRows][kGqCols / 8];
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int64_t c0 = (int64_t)blockIdx.x * kGqCols + lane * 16;
+  const int64_t row0 = (int64_t)blockIdx.y * kGqRows;
+  const bool col_ok = c0 < C1;
+  const int lanes_per_group = group >> 4;
+  const float qmax_f = (float)qmax;
+  const float tie_lim = 0.5f - tie_eps;
+  const int k_begin = blockIdx.z * k_per_cta;
+  const int k_end = min(K, k_begin + k_per_cta);
+
+#pragma unroll
+  for (int p = 0; p < kGqRows / 8; ++p) {
+    const int r = p * 8 + warp;
+    uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0;
+    if (col_ok && row0 + r < C2) {
+      const uint16_t* src = W + (row0 + r) * C1 + c0;
+      v0 = ld_nc_16(src);
+      v1 = ld_nc_16(src + 8);
+    }
+    tile[r][lane * 2] = v0;
+    tile[r][lane * 2 + 1] = v1;
+  }
+  __syncthreads();
+
+  const float2 magic2 = make_float2(kMagic, kMagic);
+  for (int k = k_begin; k < k_end; ++k) {
+    float2 sv[8], rsv[8];
+    if (!col_ok) {          // lanes past the last channel work on zeros and store nothing
+#pragma unroll
+      for (int j = 0; j < 8; ++j) sv[j] = rsv[j] = make_float2(1.0f, 1.0f);
+    } else {
+      const uint4* sp = reinterpret_cast<const uint4*>(s_tab + (int64_t)k * C1 + c0);
+      const uint4 a = sp[0], b = sp[1];
+      sv[0] = unpack2(a.x); sv[1] = unpack2(a.y); sv[2] = unpack2(a.z); sv[3] = unpack2(a.w);
+      sv[4] = unpack2(b.x); sv[5] = unpack2(b.y); sv[6] = unpack2(b.z); sv[7] = unpack2(b.w);
+      const float4* rp = reinterpret_cast<const float4*>(rs_tab + (int64_t)k * C1 + c0);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float4 r4 = rp[j];
+        rsv[2 * j] = make_float2(r4.x, r4.y);
+        rsv[2 * j + 1] = make_float2(r4.z, r4.w);
+      }
+    }
+#pragma unroll 1
+    for (int p = 0; p < kGqRows / 8; ++p) {
+      const int r = p * 8 + warp;
+      const int64_t row = row0 + r;
+      if (row >= C2) break;                       // rows of a warp ascend with p; shuffles below stay warp-uniform
+      const uint4 t0 = tile[r][lane * 2], t1 = tile[r][lane * 2 + 1];
+      float2 w[8];
+      w[0] = unpack2(t0.x); w[1] = unpack2(t0.y); w[2] = unpack2(t0.z); w[3] = unpack2(t0.w);
+      w[4] = unpack2(t1.x); w[5] = unpack2(t1.y); w[6] = unpack2(t1.z); w[7] = unpack2(t1.w);
+      float mx, mn;
+      {
+        const float2 p0 = mul2(sv[0], w[0]);       // exact: 8-bit x 8-bit significands
+        mx = fmaxf(p0.x, p0.y);
+        mn = fminf(p0.x, p0.y);
+#pragma unroll
+        for (int j = 1; j < 8; ++j) {
+          const float2 pj = mul2(sv[j], w[j]);
+          mx = max3(mx, pj.x, pj.y);
+          mn = min3(mn, pj.x, pj.y);
+        }
+      }
+      for (int off = 1; off < lanes_per_group; off <<= 1) {
+        mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
+        mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, off));
+      }
+      const float range = fmaxf(__fsub_rn(mx, mn), TLQ_RANGE_FLOOR);
+      const float step = __fdiv_rn(range, qmax_f);
+      const float inv = rcp_fast(step);
+      const float qa = __fmul_rn(mn, inv), qb = __fmul_rn(mx, inv);
+      float ra = round_magic(qa), rb = round_magic(qb);
+      if (fmaxf(fabsf(__fsub_rn(qa, ra)), fabsf(__fsub_rn(qb, rb))) > tie_lim) {
+        // an extreme sits on a rounding tie (common for bf16 weights: mx == -mn puts both on +-qmax/2): decide exactly
+        ra = round_magic(__fdiv_rn(mn, step));
+        rb = round_magic(__fdiv_rn(mx, step));
+      }
+      const bool fast = ra <= 0.0f && ra >= -qmax_f && __fsub_rn(rb, ra) <= qmax_f;   // the group cannot clip
+      uint32_t outw[8];
+      if (fast) {
+        const float2 inv2 = make_float2(inv, inv), step2 = make_float2(step, step);
+        float near = 0.0f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const float2 pj = mul2(sv[j], w[j]);
+          const float2 q = mul2(pj, inv2);
+          const float2 rq = sub2(add2(q, magic2), magic2);      // rint(q), which is q - z
+          const float2 df = sub2(q, rq);
+          near = max3(near, fabsf(df.x), fabsf(df.y));
+          const float2 w_hat = mul2(mul2(rq, step2), rsv[j]);
+          const float2 d = sub2(w[j], w_hat);
+          outw[j] = pack_bf16x2(d.x, d.y);
+        }
+        if (near > tie_lim) {
+          // some element of this thread is near a tie: find the pair(s) and redo them with the exact quotient
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const float2 pj = mul2(sv[j], w[j]);
+            const float2 q = mul2(pj, inv2);
+            const float2 df = sub2(q, sub2(add2(q, magic2), magic2));
+            if (fmaxf(fabsf(df.x), fabsf(df.y)) > tie_lim) {
+              const float2 rq = make_float2(round_magic(__fdiv_rn(pj.x, step)), round_magic(__fdiv_rn(pj.y, step)));
+              const float2 d = sub2(w[j], mul2(mul2(rq, step2), rsv[j]));
+              outw[j] = pack_bf16x2(d.x, d.y);
+            }
+          }
+        }
+      }
+      uint4* dst = reinterpret_cast<uint4*>(dW + ((int64_t)k * C2 + row) * C1 + c0);
+      if (!fast) {
+        if (col_ok)
+          delta16_general(&tile[r][lane * 2], s_tab + (int64_t)k * C1 + c0, rs_tab + (int64_t)k * C1 + c0, mn, step, inv,
+                          qmax_f, dst);
+      } else if (col_ok) {
+        dst[0] = make_uint4(outw[0], outw[1], outw[2], outw[3]);
+        dst[1] = make_uint4(outw[4], outw[5], outw[6], outw[7]);
+      }
+    }
+  }
+}
 
 __global__ void __launch_bounds__(kGqThreads)
 fakequant_group_kernel(const uint16_t* __restrict__ W, const uint16_t* __restrict__ s_tab,
@@ -195,135 +400,238 @@ int launch_fakequant_group(const uint16_t* W, const uint16_t* s, const float* rs
   const int k_per_cta = (int)ceil_div(K, kchunks);
   kchunks = ceil_div(K, k_per_cta);
   dim3 grid((unsigned)ceil_div(C1, kGqCols), (unsigned)ceil_div(C2, kGqRows), (unsigned)kchunks);
+  if (dW != nullptr && s != nullptr && rs != nullptr && codes == nullptr && steps == nullptr && zeros == nullptr) {
+    // |quotient| <= qmax + 1 on the straight-line path; 4e-7 per unit covers the reciprocal (1 ulp), the product
+    // and the exact quotient's own rounding (together < 2.4e-7 relative)
+    const float tie_eps = 4.0e-7f * (float)(1 << w_bits);
+    fakequant_delta_kernel<<<grid, kGqThreads, 0, st>>>(W, s, rs, K, k_per_cta, C2, C1, group, (1 << w_bits) - 1,
+                                                        tie_eps, dW);
+    return after_launch();
+  }
   fakequant_group_kernel<<<grid, kGqThreads, 0, st>>>(W, s, rs, K, k_per_cta, C2, C1, group, (1 << w_bits) - 1, dW,
                                                      codes, steps, zeros);
   return after_launch();
 }
 
 // ------------------------------------------------------------------------------------------------
-// int8 symmetric quantization of whole rows: weights (value = scale * w, exact) or activations
-// (value = x * (1/scale), one binary32 rounding).  One CTA owns a row at a time: the bf16 row is
-// staged in shared memory, then for every candidate the row maximum is reduced and the codes are
-// written, 16 per thread per store.
+// Symmetric quantization of whole rows into int8 containers: weights per output channel
+// (value = scale * w, exact) or activations per token (value = fl32(x * (1/scale))), step =
+// max|value| / qpos, code = rint(value / step) (Sec. 2.2, first two equations; qpos = 2^(n-1) - 1).
+//
+// A row's maximum couples all of its channels, so the work is split in two fully parallel passes
+// over the same 32-row x 512-channel tiles as the group kernels, each tile staged once in shared
+// memory and re-used for every candidate:
+//   pass 1  per (candidate, row) the maximum |value| over the tile's channels -> atomic max on the
+//           float's bit pattern (non-negative floats order like integers, so the result does not
+//           depend on arrival order); a one-line kernel then turns the maxima into steps in place;
+//   pass 2  codes: straight-line packed arithmetic, rint(value * (1/step)) with the distance to the
+//           nearest integer folded into one running maximum per thread; a thread that met a
+//           near-tie redoes its 16 elements with the exact division.  No clamp is needed:
+//           |value| <= max|value| keeps |code| <= qpos.
+// `mult` below is the per-channel multiplier of one candidate: the bf16 scale for weights, the
+// binary32 reciprocal for activations (from the table, or taken here from a bf16 scale), or 1.
 // ------------------------------------------------------------------------------------------------
-constexpr int kRowThreads = 256;
+enum MultKind { kMultScale = 0, kMultRecipTable = 1, kMultRecipOfScale = 2 };
 
-template <bool kActivation>
-__device__ __forceinline__ void scaled16(const uint4* row_smem, int64_t c, const uint16_t* s_row, const float* rs_row,
-                                         float (&v)[16]) {
-  float a[8], b[8];
-  unpack8(row_smem[c >> 3], a);
-  unpack8(row_smem[(c >> 3) + 1], b);
-  if (kActivation) {
-    if (rs_row != nullptr) {
-      const float4* r4 = reinterpret_cast<const float4*>(rs_row + c);
+template <int kKind>
+__device__ __forceinline__ void load_mult16(const uint16_t* s_row, const float* rs_row, int64_t c0, bool col_ok,
+                                            float2 (&m)[8]) {
+  if (!col_ok || (kKind != kMultRecipTable && s_row == nullptr)) {
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const float4 r = r4[j];
-        float* src = (j < 2) ? a : b;
-        const int o = (j & 1) * 4;
-        v[j * 4 + 0] = __fmul_rn(src[o + 0], r.x); v[j * 4 + 1] = __fmul_rn(src[o + 1], r.y);
-        v[j * 4 + 2] = __fmul_rn(src[o + 2], r.z); v[j * 4 + 3] = __fmul_rn(src[o + 3], r.w);
-      }
-    } else if (s_row != nullptr) {      // single scale vector given as bf16: take the reciprocal here
-      float sa[8], sb[8];
-      unpack8(*reinterpret_cast<const uint4*>(s_row + c), sa);
-      unpack8(*reinterpret_cast<const uint4*>(s_row + c + 8), sb);
+    for (int j = 0; j < 8; ++j) m[j] = make_float2(1.0f, 1.0f);
+    return;
+  }
+  if (kKind == kMultRecipTable) {
+    const float4* rp = reinterpret_cast<const float4*>(rs_row + c0);
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        v[j] = __fmul_rn(a[j], __fdiv_rn(1.0f, sa[j]));
-        v[8 + j] = __fmul_rn(b[j], __fdiv_rn(1.0f, sb[j]));
-      }
-    } else {
-#pragma unroll
-      for (int j = 0; j < 8; ++j) { v[j] = a[j]; v[8 + j] = b[j]; }
+    for (int j = 0; j < 4; ++j) {
+      const float4 r4 = rp[j];
+      m[2 * j] = make_float2(r4.x, r4.y);
+      m[2 * j + 1] = make_float2(r4.z, r4.w);
     }
   } else {
-    if (s_row != nullptr) {
-      float sa[8], sb[8];
-      unpack8(*reinterpret_cast<const uint4*>(s_row + c), sa);
-      unpack8(*reinterpret_cast<const uint4*>(s_row + c + 8), sb);
+    const uint4* sp = reinterpret_cast<const uint4*>(s_row + c0);
+    const uint4 a = sp[0], b = sp[1];
+    m[0] = unpack2(a.x); m[1] = unpack2(a.y); m[2] = unpack2(a.z); m[3] = unpack2(a.w);
+    m[4] = unpack2(b.x); m[5] = unpack2(b.y); m[6] = unpack2(b.z); m[7] = unpack2(b.w);
+    if (kKind == kMultRecipOfScale) {
 #pragma unroll
-      for (int j = 0; j < 8; ++j) { v[j] = __fmul_rn(sa[j], a[j]); v[8 + j] = __fmul_rn(sb[j], b[j]); }
-    } else {
-#pragma unroll
-      for (int j = 0; j < 8; ++j) { v[j] = a[j]; v[8 + j] = b[j]; }
+      for (int j = 0; j < 8; ++j) m[j] = make_float2(__fdiv_rn(1.0f, m[j].x), __fdiv_rn(1.0f, m[j].y));
     }
   }
 }
 
-template <bool kActivation>
-__global__ void __launch_bounds__(kRowThreads)
-quant_rows_i8_kernel(const uint16_t* __restrict__ src, const uint16_t* __restrict__ s_tab,
-                     const float* __restrict__ rs_tab, int K, int64_t R, int64_t C1, int8_t* __restrict__ q,
-                     float* __restrict__ step_out) {
-  extern __shared__ uint4 row_smem[];      // C1/8 packets
-  __shared__ float warp_max[2][kRowThreads / 32];
-  const int t = threadIdx.x;
-  for (int64_t row = blockIdx.x; row < R; row += gridDim.x) {
-    __syncthreads();
-    for (int64_t i = t; i < C1 / 8; i += kRowThreads) row_smem[i] = ld_nc_16(src + row * C1 + i * 8);
-    __syncthreads();
-    for (int k = 0; k < K; ++k) {
-      const uint16_t* s_row = (s_tab != nullptr) ? s_tab + (int64_t)k * C1 : nullptr;
-      const float* rs_row = (rs_tab != nullptr) ? rs_tab + (int64_t)k * C1 : nullptr;
-      float amax = 0.0f;
-      for (int64_t c = (int64_t)t * 16; c < C1; c += kRowThreads * 16) {
-        float v[16];
-        scaled16<kActivation>(row_smem, c, s_row, rs_row, v);
+__device__ __forceinline__ void stage_tile(uint4 (*tile)[kGqCols / 8], const uint16_t* __restrict__ src, int64_t row0,
+                                           int64_t R, int64_t C1, int64_t c0, bool col_ok, int warp, int lane) {
 #pragma unroll
-        for (int j = 0; j < 16; ++j) amax = fmaxf(amax, fabsf(v[j]));
+  for (int p = 0; p < kGqRows / 8; ++p) {
+    const int r = p * 8 + warp;
+    uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0;
+    if (col_ok && row0 + r < R) {
+      const uint16_t* sp = src + (row0 + r) * C1 + c0;
+      v0 = ld_nc_16(sp);
+      v1 = ld_nc_16(sp + 8);
+    }
+    tile[r][lane * 2] = v0;
+    tile[r][lane * 2 + 1] = v1;
+  }
+  __syncthreads();
+}
+
+__device__ __forceinline__ void unpack16(const uint4& t0, const uint4& t1, float2 (&w)[8]) {
+  w[0] = unpack2(t0.x); w[1] = unpack2(t0.y); w[2] = unpack2(t0.z); w[3] = unpack2(t0.w);
+  w[4] = unpack2(t1.x); w[5] = unpack2(t1.y); w[6] = unpack2(t1.z); w[7] = unpack2(t1.w);
+}
+
+template <int kKind>
+__global__ void __launch_bounds__(kGqThreads, 3)
+row_amax_kernel(const uint16_t* __restrict__ src, const uint16_t* __restrict__ s_tab, const float* __restrict__ rs_tab,
+                int K, int k_per_cta, int64_t R, int64_t C1, int* __restrict__ amax_bits /*[K,R], zeroed*/) {
+  __shared__ uint4 tile[kGqRows][kGqCols / 8];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t c0 = (int64_t)blockIdx.x * kGqCols + lane * 16;
+  const int64_t row0 = (int64_t)blockIdx.y * kGqRows;
+  const bool col_ok = c0 < C1;
+  stage_tile(tile, src, row0, R, C1, c0, col_ok, warp, lane);
+  const int k_begin = blockIdx.z * k_per_cta;
+  const int k_end = min(K, k_begin + k_per_cta);
+  for (int k = k_begin; k < k_end; ++k) {
+    float2 m[8];
+    load_mult16<kKind>(s_tab ? s_tab + (int64_t)k * C1 : nullptr, rs_tab ? rs_tab + (int64_t)k * C1 : nullptr, c0,
+                       col_ok, m);
+#pragma unroll 1
+    for (int p = 0; p < kGqRows / 8; ++p) {
+      const int r = p * 8 + warp;
+      if (row0 + r >= R) break;
+      float2 w[8];
+      unpack16(tile[r][lane * 2], tile[r][lane * 2 + 1], w);
+      float a = 0.0f;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const float2 v = mul2(w[j], m[j]);
+        a = max3(a, fabsf(v.x), fabsf(v.y));
       }
 #pragma unroll
-      for (int off = 16; off > 0; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, off));
-      float* wm = warp_max[k & 1];          // double-buffered: one barrier per candidate
-      if ((t & 31) == 0) wm[t >> 5] = amax;
-      __syncthreads();
-      float m = wm[0];
+      for (int off = 16; off > 0; off >>= 1) a = fmaxf(a, __shfl_xor_sync(0xFFFFFFFFu, a, off));
+      if (lane == 0) atomicMax(amax_bits + (int64_t)k * R + row0 + r, __float_as_int(a));
+    }
+  }
+}
+
+__global__ void amax_to_step_kernel(float* __restrict__ v, int64_t n, float qpos) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) v[i] = __fdiv_rn(fmaxf(v[i], TLQ_RANGE_FLOOR), qpos);
+}
+
+// One thread's 16 codes with the exact division (a near-tie was seen on the straight-line path).
+__device__ __noinline__ void codes16_exact(const uint4* tile16, const float* mult16, float st, float qpos, uint4* dst) {
+  uint32_t pk[4] = {0u, 0u, 0u, 0u};
+#pragma unroll 1
+  for (int h = 0; h < 2; ++h) {
+    float w[8];
+    unpack8(tile16[h], w);
 #pragma unroll
-      for (int w = 1; w < kRowThreads / 32; ++w) m = fmaxf(m, wm[w]);
-      const float st = __fdiv_rn(fmaxf(m, TLQ_RANGE_FLOOR), 127.0f);
+    for (int j = 0; j < 8; ++j) {
+      const float v = __fmul_rn(w[j], mult16[h * 8 + j]);
+      const float q = fminf(fmaxf(__fdiv_rn(v, st), -qpos - 1.0f), qpos);
+      const int e = h * 8 + j;
+      pk[e >> 2] |= (__float_as_uint(__fadd_rn(q, kMagic)) & 0xFFu) << ((e & 3) * 8);
+    }
+  }
+  *dst = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+}
+
+template <int kKind>
+__global__ void __launch_bounds__(kGqThreads, 3)
+row_codes_kernel(const uint16_t* __restrict__ src, const uint16_t* __restrict__ s_tab, const float* __restrict__ rs_tab,
+                 const float* __restrict__ step /*[K,R]*/, int K, int k_per_cta, int64_t R, int64_t C1, float qpos,
+                 float tie_eps, int8_t* __restrict__ q /*[K,R,C1]*/) {
+  __shared__ uint4 tile[kGqRows][kGqCols / 8];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t c0 = (int64_t)blockIdx.x * kGqCols + lane * 16;
+  const int64_t row0 = (int64_t)blockIdx.y * kGqRows;
+  const bool col_ok = c0 < C1;
+  stage_tile(tile, src, row0, R, C1, c0, col_ok, warp, lane);
+  if (!col_ok) return;                    // no warp-wide operation below
+  const float tie_lim = 0.5f - tie_eps;
+  const float2 magic2 = make_float2(kMagic, kMagic);
+  const int k_begin = blockIdx.z * k_per_cta;
+  const int k_end = min(K, k_begin + k_per_cta);
+  for (int k = k_begin; k < k_end; ++k) {
+    float2 m[8];
+    load_mult16<kKind>(s_tab ? s_tab + (int64_t)k * C1 : nullptr, rs_tab ? rs_tab + (int64_t)k * C1 : nullptr, c0,
+                       true, m);
+#pragma unroll 1
+    for (int p = 0; p < kGqRows / 8; ++p) {
+      const int r = p * 8 + warp;
+      const int64_t row = row0 + r;
+      if (row >= R) break;
+      const float st = step[(int64_t)k * R + row];
       const float inv = rcp_fast(st);
-      if (t == 0) step_out[(int64_t)k * R + row] = st;
-      int8_t* out = q + ((int64_t)k * R + row) * C1;
-      for (int64_t c = (int64_t)t * 16; c < C1; c += kRowThreads * 16) {
-        float v[16];
-        scaled16<kActivation>(row_smem, c, s_row, rs_row, v);
-        uint32_t pk[4] = {0u, 0u, 0u, 0u};
+      const float2 inv2 = make_float2(inv, inv);
+      float2 w[8];
+      unpack16(tile[r][lane * 2], tile[r][lane * 2 + 1], w);
+      float near = 0.0f;
+      uint32_t tb[16];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const float qi = quotient_rint_clamped(v[j], st, inv, -128.0f, 127.0f);
-          pk[j >> 2] |= (__float_as_uint(__fadd_rn(qi, kMagic)) & 0xFFu) << ((j & 3) * 8);
-        }
-        *reinterpret_cast<uint4*>(out + c) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+      for (int j = 0; j < 8; ++j) {
+        const float2 qv = mul2(mul2(w[j], m[j]), inv2);
+        const float2 t = add2(qv, magic2);           // low mantissa byte = the code in two's complement
+        const float2 df = sub2(qv, sub2(t, magic2));
+        near = max3(near, fabsf(df.x), fabsf(df.y));
+        tb[2 * j] = __float_as_uint(t.x);
+        tb[2 * j + 1] = __float_as_uint(t.y);
+      }
+      uint4* dst = reinterpret_cast<uint4*>(q + ((int64_t)k * R + row) * C1 + c0);
+      if (near > tie_lim) {
+        float mf[16];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { mf[2 * j] = m[j].x; mf[2 * j + 1] = m[j].y; }
+        codes16_exact(&tile[r][lane * 2], mf, st, qpos, dst);
+      } else {
+        uint32_t pk[4];
+#pragma unroll
+        for (int g = 0; g < 4; ++g)
+          pk[g] = __byte_perm(__byte_perm(tb[4 * g], tb[4 * g + 1], 0x0040), __byte_perm(tb[4 * g + 2], tb[4 * g + 3], 0x0040),
+                              0x5410);
+        *dst = make_uint4(pk[0], pk[1], pk[2], pk[3]);
       }
     }
   }
 }
 
-template <bool kActivation>
-static int launch_rows(const uint16_t* src, const uint16_t* s, const float* rs, int K, int64_t R, int64_t C1,
+template <int kKind>
+static int launch_rows(const uint16_t* src, const uint16_t* s, const float* rs, int K, int64_t R, int64_t C1, int bits,
                        int8_t* q, float* step, cudaStream_t st) {
-  const size_t smem = (size_t)C1 * 2;
-  static bool configured = false;
-  if (!configured) {
-    TLQ_CUDA_TRY(cudaFuncSetAttribute(quant_rows_i8_kernel<kActivation>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      200 * 1024));
-    configured = true;
-  }
-  int64_t grid = R < 148 * 8 ? R : 148 * 8;
-  quant_rows_i8_kernel<kActivation><<<(unsigned)grid, kRowThreads, smem, st>>>(src, s, rs, K, R, C1, q, step);
+  const int64_t ctas = ceil_div(C1, kGqCols) * ceil_div(R, kGqRows);
+  int64_t kchunks = ceil_div(148 * 6, ctas);
+  if (kchunks > K) kchunks = K;
+  if (kchunks < 1) kchunks = 1;
+  const int k_per_cta = (int)ceil_div(K, kchunks);
+  kchunks = ceil_div(K, k_per_cta);
+  const dim3 grid((unsigned)ceil_div(C1, kGqCols), (unsigned)ceil_div(R, kGqRows), (unsigned)kchunks);
+  const float qpos = (float)((1 << (bits - 1)) - 1);
+  const float tie_eps = 4.0e-7f * (qpos + 1.0f);
+  const int64_t n = (int64_t)K * R;
+  TLQ_CUDA_TRY(cudaMemsetAsync(step, 0, (size_t)n * sizeof(float), st));
+  row_amax_kernel<kKind><<<grid, kGqThreads, 0, st>>>(src, s, rs, K, k_per_cta, R, C1, reinterpret_cast<int*>(step));
+  int rc = after_launch();
+  if (rc != TLQ_OK) return rc;
+  amax_to_step_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(step, n, qpos);
+  if ((rc = after_launch()) != TLQ_OK) return rc;
+  row_codes_kernel<kKind><<<grid, kGqThreads, 0, st>>>(src, s, rs, step, K, k_per_cta, R, C1, qpos, tie_eps, q);
   return after_launch();
 }
 
-int launch_fakequant_rows_i8(const uint16_t* W, const uint16_t* s, int K, int64_t C2, int64_t C1, int8_t* q, float* u,
-                             cudaStream_t st) {
-  return launch_rows<false>(W, s, nullptr, K, C2, C1, q, u, st);
+int launch_fakequant_rows_i8(const uint16_t* W, const uint16_t* s, int K, int64_t C2, int64_t C1, int bits, int8_t* q,
+                             float* u, cudaStream_t st) {
+  return launch_rows<kMultScale>(W, s, nullptr, K, C2, C1, bits, q, u, st);
 }
 
-int launch_actquant_i8(const uint16_t* X, const uint16_t* s, const float* rs, int K, int64_t N, int64_t C1, int8_t* q,
-                       float* t, cudaStream_t st) {
-  return launch_rows<true>(X, s, rs, K, N, C1, q, t, st);
+int launch_actquant_i8(const uint16_t* X, const uint16_t* s, const float* rs, int K, int64_t N, int64_t C1, int bits,
+                       int8_t* q, float* t, cudaStream_t st) {
+  if (rs != nullptr) return launch_rows<kMultRecipTable>(X, nullptr, rs, K, N, C1, bits, q, t, st);
+  return launch_rows<kMultRecipOfScale>(X, s, nullptr, K, N, C1, bits, q, t, st);
 }
 
 }  // namespace tlq

@@ -42,6 +42,8 @@ struct GemmArgs {
   int num_kb;              // ceil(C1 / 64)
   int64_t mtiles, otiles;
   int64_t num_tiles;       // K * otiles * mtiles
+  int64_t tiles_per_k;     // otiles * mtiles
+  TileRaster raster;       // walk order inside one candidate
   int64_t n_pad;
   const float* w_imp;      // [N] or null (uniform)
   float* partials;         // [K][otiles*mtiles*4]
@@ -104,10 +106,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       uint32_t phase = 0;
       bool ok = true;
       for (int64_t tile = blockIdx.x; tile < args.num_tiles && ok; tile += gridDim.x) {
-        const int64_t mt = tile % args.mtiles;
-        const int64_t rest = tile / args.mtiles;
-        const int ot = (int)(rest % args.otiles);
-        const int k = (int)(rest / args.otiles);
+        const int k = (int)(tile / args.tiles_per_k);
+        int mt, ot;
+        args.raster.decode(tile - (int64_t)k * args.tiles_per_k, mt, ot);
         for (int pass = 0; pass < passes && ok; ++pass) {
           const CUtensorMap* tb = (kApply && pass == 1) ? &tmB2 : &tmB;
           for (int kb = 0; kb < num_kb; ++kb) {
@@ -118,7 +119,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             }
             const uint32_t a_dst = smem_base + stage * kStageBytes;
             ptx::mbar_expect_tx(full_bar(stage), kStageBytes);
-            ptx::tma_load_2d(a_dst, &tmA, full_bar(stage), kb * BK, (int)(mt * BM));
+            ptx::tma_load_2d(a_dst, &tmA, full_bar(stage), kb * BK, mt * BM);
             ptx::tma_load_3d(a_dst + kABytes, tb, full_bar(stage), kb * BK, ot * BN, k);
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
           }
@@ -173,10 +174,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int row_in_tile = quarter * 32 + lane;
     int64_t it = 0;
     for (int64_t tile = blockIdx.x; tile < args.num_tiles; tile += gridDim.x, ++it) {
-      const int64_t mt = tile % args.mtiles;
-      const int64_t rest = tile / args.mtiles;
-      const int ot = (int)(rest % args.otiles);
-      const int k = (int)(rest / args.otiles);
+      const int k = (int)(tile / args.tiles_per_k);
+      int mt, ot;
+      args.raster.decode(tile - (int64_t)k * args.tiles_per_k, mt, ot);
       const int acc = (int)(it & 1);
       const uint32_t acc_phase = (uint32_t)((it >> 1) & 1);
       if (!ptx::mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) {
@@ -185,7 +185,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       }
       ptx::tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * BN;
-      const int64_t n = mt * BM + row_in_tile;
+      const int64_t n = (int64_t)mt * BM + row_in_tile;
       if (!kApply) {
         float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll 1
@@ -336,12 +336,14 @@ int launch_search_gemm_bf16(const uint16_t* X, const uint16_t* dW, const float* 
   a.N = plan.N; a.C2 = plan.C2;
   a.num_kb = (int)ceil_div(plan.C1, BK);
   a.mtiles = plan.mtiles; a.otiles = plan.otiles;
-  a.num_tiles = (int64_t)plan.K * plan.otiles * plan.mtiles;
+  a.tiles_per_k = plan.otiles * plan.mtiles;
+  a.num_tiles = (int64_t)plan.K * a.tiles_per_k;
   a.n_pad = plan.n_pad;
   a.w_imp = w_imp; a.partials = partials; a.ptab = ptab; a.bias = nullptr; a.yq = nullptr; a.hdr = hdr;
   const int sms = num_sms();
   if (sms <= 0) return TLQ_ERR_CUDA;
   const unsigned grid = (unsigned)(a.num_tiles < sms ? a.num_tiles : sms);
+  a.raster = make_raster(plan.mtiles, plan.otiles, sms, plan.N * plan.C1 * 2);
   gemm_bf16_kernel<false><<<grid, kThreads, kSmemBytes, st>>>(tmA, tmB, tmB, a);
   return after_launch();
 }
@@ -358,12 +360,14 @@ int launch_apply_gemm_bf16(const uint16_t* X, const uint16_t* W, const uint16_t*
   a.N = N; a.C2 = C2;
   a.num_kb = (int)ceil_div(C1, BK);
   a.mtiles = plan.mtiles; a.otiles = plan.otiles;
-  a.num_tiles = plan.otiles * plan.mtiles;
+  a.tiles_per_k = plan.otiles * plan.mtiles;
+  a.num_tiles = a.tiles_per_k;
   a.n_pad = plan.n_pad;
   a.w_imp = nullptr; a.partials = nullptr; a.ptab = nullptr; a.bias = bias; a.yq = Yq; a.hdr = hdr;
   const int sms = num_sms();
   if (sms <= 0) return TLQ_ERR_CUDA;
   const unsigned grid = (unsigned)(a.num_tiles < sms ? a.num_tiles : sms);
+  a.raster = make_raster(plan.mtiles, plan.otiles, sms, plan.N * plan.C1 * 2);
   gemm_bf16_kernel<true><<<grid, kThreads, kSmemBytes, st>>>(tmA, tmW, tmD, a);
   return after_launch();
 }

@@ -47,6 +47,7 @@ struct I8Args {
   int K;
   int64_t mtiles, otiles;
   int64_t num_tiles;       // otiles * mtiles (every tile runs all passes)
+  TileRaster raster;       // walk order of the tiles
   int64_t n_pad;
   const float* w_imp;      // [N] or null
   const float* t;          // [K,N] activation steps
@@ -113,8 +114,8 @@ gemm_w8a8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       uint32_t phase = 0;
       bool ok = true;
       for (int64_t tile = blockIdx.x; tile < args.num_tiles && ok; tile += gridDim.x) {
-        const int mt = (int)(tile % args.mtiles);
-        const int ot = (int)(tile / args.mtiles);
+        int mt, ot;
+        args.raster.decode(tile, mt, ot);
         for (int pass = 0; pass < passes && ok; ++pass) {
           const bool fp = !kApply && pass == 0;
           const int k = kApply ? 0 : pass - 1;
@@ -194,10 +195,10 @@ gemm_w8a8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     int64_t it = 0;
     bool ok = true;
     for (int64_t tile = blockIdx.x; tile < args.num_tiles && ok; tile += gridDim.x) {
-      const int64_t mt = tile % args.mtiles;
-      const int64_t ot = tile / args.mtiles;
-      const int64_t n = mt * BM + row_in_tile;
-      const int64_t col_base = ot * BN + half * 128;
+      int mt, ot;
+      args.raster.decode(tile, mt, ot);
+      const int64_t n = (int64_t)mt * BM + row_in_tile;
+      const int64_t col_base = (int64_t)ot * BN + half * 128;
       for (int pass = 0; pass < passes; ++pass, ++it) {
         const int acc = (int)(it & 1);
         const uint32_t acc_phase = (uint32_t)((it >> 1) & 1);
@@ -257,7 +258,7 @@ gemm_w8a8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
 #pragma unroll
           for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
           if (lane == 0)
-            args.partials[(int64_t)k * args.otiles * args.mtiles * 8 + (ot * args.mtiles + mt) * 8 + ew] = v;
+            args.partials[(int64_t)k * args.otiles * args.mtiles * 8 + ((int64_t)ot * args.mtiles + mt) * 8 + ew] = v;
         } else {
 #pragma unroll 1
           for (int c = 0; c < 8; ++c) {
@@ -372,6 +373,7 @@ int launch_search_gemm_i8(const uint16_t* X, const uint16_t* W, const int8_t* Xq
   const int sms = sm_count();
   if (sms <= 0) return TLQ_ERR_CUDA;
   const unsigned grid = (unsigned)(a.num_tiles < sms ? a.num_tiles : sms);
+  a.raster = make_raster(plan.mtiles, plan.otiles, sms, plan.N * plan.C1);
   gemm_w8a8_kernel<false><<<grid, kThreads, kSmemBytes, st>>>(tmX, tmW, tmXq, tmWq, a);
   return after_launch();
 }
@@ -395,6 +397,7 @@ int launch_apply_gemm_i8(const int8_t* Xq, const int8_t* Wq, const float* t, con
   const int sms = sm_count();
   if (sms <= 0) return TLQ_ERR_CUDA;
   const unsigned grid = (unsigned)(a.num_tiles < sms ? a.num_tiles : sms);
+  a.raster = make_raster(plan.mtiles, plan.otiles, sms, plan.N * plan.C1);
   gemm_w8a8_kernel<true><<<grid, kThreads, kSmemBytes, st>>>(tmXq, tmWq, tmXq, tmWq, a);
   return after_launch();
 }
