@@ -181,8 +181,11 @@ def run_ours(args, cfgw):
     cfgr = dataclasses.replace(cfgw, seed=replicas.replica_seed(cfgw.seed, rank))
     data = wl.LayerData(cfgr)
     lins = [l for l in cfgr.linears() if args.linears is None or l.name in args.linears.split(",")]
-    mode = tlq.W4A16_ASYM_GROUP if cfgr.mode == "w4a16" else tlq.W8A8_SYM
-    cfg = tlq.config(mode=mode, group_size=cfgr.group, n_grid=cfgr.n_grid)
+    if cfgr.mode == "w4a16":
+        cfg = tlq.config(mode=tlq.W4A16_ASYM_GROUP, group_size=cfgr.group, n_grid=cfgr.n_grid)
+    else:   # "w<n>a<m>": symmetric per-channel weights / per-token activations on the int8 tensor-core path
+        wn, an = (int(v) for v in cfgr.mode[1:].split("a"))
+        cfg = tlq.config(mode=tlq.WA_SYM_CHANNEL, w_bits=wn, a_bits=an, n_grid=cfgr.n_grid)
 
     # host (pinned) copies for the end-to-end leg, device-resident copies for the kernel leg
     host_x, host_w, dev_x, dev_w = {}, {}, {}, {}
@@ -362,12 +365,13 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="cfg1")
+    ap.add_argument("--mode", default=None, help="override the config's setting: w4a16, w8a8, w4a8, w4a6")
     ap.add_argument("--linears", default=None, help="comma-separated subset of q,k,v,o,gate,up,down (profiling)")
     ap.add_argument("--profile", action="store_true", help="kernel leg only: skip the end-to-end and CPU legs")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     from paper_2602_07899_b200 import workloads as wl
-    cfgw = wl.config(args.config)
+    cfgw = wl.config(args.config) if args.mode is None else wl.config(args.config, mode=args.mode)
     if args.impl == "reference":
         run_reference(args, cfgw)
     else:

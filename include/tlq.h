@@ -46,8 +46,12 @@ extern "C" {
 #define TLQ_W4A16_ASYM_GROUP 0 /* weights: w_bits (2..8) asymmetric, one step + integer zero-point per
                                   `group_size` consecutive input channels of an output row; activations
                                   stay bf16 (Q_a = identity) */
-#define TLQ_W8A8_SYM 1         /* weights: int8 symmetric per output row; activations: int8 symmetric per
-                                  token, both with step max|.|/127 (Sec. 2.2, first two equations) */
+#define TLQ_W8A8_SYM 1         /* weights: w_bits (2..8) symmetric per output row; activations: a_bits (2..8)
+                                  symmetric per token; step max|.|/(2^(bits-1)-1), integers in
+                                  [-2^(bits-1), 2^(bits-1)-1] held in int8 containers (Sec. 2.2, first two
+                                  equations).  w_bits = a_bits = 8 is W8A8; the paper's main settings are
+                                  w_bits = 4 with a_bits = 8 or 6 (Experiments, quantization settings) */
+#define TLQ_WA_SYM_CHANNEL TLQ_W8A8_SYM /* the same mode under the name of what it does */
 
 /* tlq_config.stat_mode: x_stat over the calibration tokens */
 #define TLQ_STAT_MEAN_ABS 0   /* mean_n |X_nc| (x_mean row of the paper's ablation table) */
@@ -65,8 +69,8 @@ extern "C" {
 typedef struct {
   uint32_t struct_size; /* sizeof(tlq_config); checked */
   int32_t mode;         /* TLQ_W4A16_ASYM_GROUP | TLQ_W8A8_SYM */
-  int32_t w_bits;       /* 2..8 for the group mode (codes are one per byte), 8 for W8A8 */
-  int32_t a_bits;       /* 16 for the group mode, 8 for W8A8 */
+  int32_t w_bits;       /* 2..8 (codes are one per byte in both modes) */
+  int32_t a_bits;       /* 16 for the group mode; 2..8 for the symmetric mode */
   int32_t group_size;   /* 32, 64, 128 or 256 for the group mode (must divide C1); ignored for W8A8 */
   int32_t n_grid;       /* K >= 1; candidate k uses r_k = k / K, so candidate 0 is scale = 1 */
   int32_t stat_mode;    /* TLQ_STAT_* */
@@ -133,15 +137,15 @@ int tlq_scale_candidates_noalloc(const void* X, int64_t N, int64_t C1, const uin
  *   W [C2,C1] bf16;  s [C1] bf16 or NULL (= all ones, plain round-to-nearest)
  * Group mode: codes [C2,C1] uint8 in [0,2^w_bits-1]; steps [C2,C1/G] fp32; zeros [C2,C1/G] int32;
  *             dW_out [C2,C1] bf16 or NULL: W - dequant/scale (the tensor-core operand of the search).
- * W8A8 mode:  codes [C2,C1] int8 bits; steps [C2] fp32; zeros ignored (may be NULL); dW_out must be NULL.
+ * Symmetric mode: codes [C2,C1] int8 (w_bits wide); steps [C2] fp32; zeros ignored (may be NULL); dW_out must be NULL.
  * Any of codes/steps/zeros may be NULL when not wanted.
  */
 int tlq_quantize_weights(const void* W, const void* s, int64_t C2, int64_t C1, const tlq_config* cfg,
                          uint8_t* codes, float* steps, int32_t* zeros, void* dW_out, void* stream);
 
 /*
- * Quantize the smoothed activations for ONE scale vector: Q_a(x / scale), per-token symmetric int8
- * (Sec. 2.2 first two equations; Sec. 3.2.1 f_q).  W8A8 mode only.
+ * Quantize the smoothed activations for ONE scale vector: Q_a(x / scale), per-token symmetric, a_bits wide
+ * (Sec. 2.2 first two equations; Sec. 3.2.1 f_q).  Symmetric mode only.
  *   X [N,C1] bf16; s [C1] bf16 or NULL (= ones); codes [N,C1] int8; steps [N] fp32.
  */
 int tlq_quantize_activations(const void* X, const void* s, int64_t N, int64_t C1, const tlq_config* cfg,

@@ -78,16 +78,19 @@ def search(x_bits, w_bits, w_imp, group: int, n_grid: int, bits: int = 4, mode: 
                 for o in range(c2):
                     y_q[i][o] = sum(w_hat[o][c] * x[i][c] for c in range(c1))
         else:
+            # "w<n>a<m>": symmetric, step = max|.| / (2^(bits-1) - 1), integers in [-2^(bits-1), 2^(bits-1)-1]
+            wn, an = (int(v) for v in mode[1:].split("a"))
+            wpos, apos = (1 << (wn - 1)) - 1, (1 << (an - 1)) - 1
             qw, u = [], []
             for o in range(c2):
                 p = [f32(w[o][c] * s[c]) for c in range(c1)]
-                uo = f32(max(max(abs(v) for v in p), f32(1e-5)) / 127.0)
+                uo = f32(max(max(abs(v) for v in p), f32(1e-5)) / float(wpos))
                 u.append(uo)
-                qw.append([min(max(round_half_even(f32(v / uo)), -128), 127) for v in p])
+                qw.append([min(max(round_half_even(f32(v / uo)), -wpos - 1), wpos) for v in p])
             for i in range(n):
                 xt = [f32(x[i][c] * f32(1.0 / s[c])) for c in range(c1)]
-                t = f32(max(max(abs(v) for v in xt), f32(1e-5)) / 127.0)
-                qx = [min(max(round_half_even(f32(v / t)), -128), 127) for v in xt]
+                t = f32(max(max(abs(v) for v in xt), f32(1e-5)) / float(apos))
+                qx = [min(max(round_half_even(f32(v / t)), -apos - 1), apos) for v in xt]
                 for o in range(c2):
                     y_q[i][o] = t * u[o] * sum(qx[c] * qw[o][c] for c in range(c1))
         e = [sum((y_fp[i][o] - y_q[i][o]) ** 2 for o in range(c2)) for i in range(n)]

@@ -239,20 +239,34 @@ def argmin_lowest(losses: np.ndarray) -> int:
     return idx
 
 
+def symmetric_bits(mode: str) -> tuple[int, int]:
+    """(weight bits, activation bits) of a per-channel / per-token symmetric setting named "w<n>a<m>":
+    "w8a8", and the paper's main settings "w4a8" and "w4a6" (Experiments, quantization settings:
+    per-token symmetric activations, per-channel symmetric weights)."""
+    if not (mode.startswith("w") and "a" in mode[1:]):
+        raise ValueError(mode)
+    n, m = mode[1:].split("a", 1)
+    n, m = int(n), int(m)
+    if not (2 <= n <= 8 and 2 <= m <= 8):
+        raise ValueError(mode)
+    return n, m
+
+
 def candidate_error(x_bits, w_bits, s_k, mode: str, group: int, y_fp: np.ndarray | None = None,
-                    w_bits_n: int = 4, a_bits_n: int = 8) -> np.ndarray:
-    """Per-token squared output error of one scale candidate, float64 [N]."""
+                    w_bits_n: int = 4) -> np.ndarray:
+    """Per-token squared output error of one scale candidate, float64 [N].
+    mode "w4a16": group-wise asymmetric `w_bits_n`-bit weights, activations untouched;
+    mode "w<n>a<m>" otherwise: symmetric n-bit weights per output channel, m-bit activations per token."""
     if y_fp is None:
         y_fp = layer_fp(x_bits, w_bits)
     if mode == "w4a16":
         _, _, _, w_hat = quantize_weights_group_asym(w_bits, s_k, group, w_bits_n)
         y_q = layer_q_w4a16(x_bits, w_hat)
-    elif mode == "w8a8":
-        qw, u = quantize_weights_row_sym(w_bits, s_k, 8)
-        qx, t = quantize_activations_token_sym(x_bits, s_k, a_bits_n)
-        y_q = layer_q_w8a8(qx, t, qw, u)
     else:
-        raise ValueError(mode)
+        wn, an = symmetric_bits(mode)
+        qw, u = quantize_weights_row_sym(w_bits, s_k, wn)
+        qx, t = quantize_activations_token_sym(x_bits, s_k, an)
+        y_q = layer_q_w8a8(qx, t, qw, u)
     return per_token_error(y_fp, y_q)
 
 
@@ -285,8 +299,9 @@ def apply_layer(x_bits, w_bits, s, bias_bits, mode: str = "w4a16", group: int = 
     if mode == "w4a16":
         codes, step, zero, w_hat = quantize_weights_group_asym(w_bits, s, group, w_bits_n)
         return layer_q_w4a16(x_bits, w_hat, b), (codes, step, zero)
-    qw, u = quantize_weights_row_sym(w_bits, s, 8)
-    qx, t = quantize_activations_token_sym(x_bits, s, 8)
+    wn, an = symmetric_bits(mode)
+    qw, u = quantize_weights_row_sym(w_bits, s, wn)
+    qx, t = quantize_activations_token_sym(x_bits, s, an)
     return layer_q_w8a8(qx, t, qw, u, b), (qw, u, None)
 
 

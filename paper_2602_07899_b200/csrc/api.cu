@@ -26,8 +26,8 @@ int check_cfg(const tlq_config* cfg, int64_t C1, bool need_quantizer = true) {
     if (g != 32 && g != 64 && g != 128 && g != 256) return TLQ_ERR_UNSUPPORTED;
     if ((C1 % g) != 0) return TLQ_ERR_SHAPE;
   } else if (cfg->mode == TLQ_W8A8_SYM) {
-    if (cfg->w_bits != 8 || cfg->a_bits != 8) return TLQ_ERR_UNSUPPORTED;
-    if ((C1 % 16) != 0 || C1 * 2 > 200 * 1024) return TLQ_ERR_SHAPE;
+    if (cfg->w_bits < 2 || cfg->w_bits > 8 || cfg->a_bits < 2 || cfg->a_bits > 8) return TLQ_ERR_UNSUPPORTED;
+    if ((C1 % 16) != 0) return TLQ_ERR_SHAPE;
   } else {
     return TLQ_ERR_INVALID_ARG;
   }

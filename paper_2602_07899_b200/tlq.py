@@ -20,6 +20,7 @@ OK = 0
 ERR_INVALID_ARG, ERR_SHAPE, ERR_ALIGN, ERR_UNSUPPORTED = -1, -2, -3, -4
 ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_NONFINITE = -5, -6, -7, -8
 W4A16_ASYM_GROUP, W8A8_SYM = 0, 1
+WA_SYM_CHANNEL = W8A8_SYM     # symmetric per-channel weights / per-token activations, w_bits and a_bits in 2..8
 STAT_MEAN_ABS, STAT_MAX_ABS, STAT_MASKED_MAX = 0, 1, 2
 NORM_MEAN_ABS, NORM_L2 = 0, 1
 DTYPE_BF16, DTYPE_F32 = 0, 1

@@ -148,7 +148,7 @@ class LayerConfig:
     visual_frac: float
     dist: str = "normal"
     n_outlier: int = 4
-    mode: str = "w4a16"       # "w4a16" | "w8a8"
+    mode: str = "w4a16"       # "w4a16" (group-wise asymmetric weights) | "w8a8", "w4a8", "w4a6" (symmetric)
     group: int = 128
     n_grid: int = 20
     imp_kind: str = "lognormal"

@@ -306,3 +306,57 @@ def test_apply_layer_w8a8(tlq):
     yq = out["Yq"].float().cpu().numpy().astype(np.float64)
     # integer accumulation is exact; what remains is the bf16 rounding of the output (2^-9 relative, doubled)
     assert np.all(np.abs(yq - yq_ref) <= 2.0 ** -8 * np.abs(yq_ref) + 1e-6)
+
+
+# ----------------------------------------------------------------------------------- W4A8 / W4A6 (the paper's settings)
+
+
+@pytest.mark.parametrize("w_bits,a_bits", [(4, 8), (4, 6), (6, 4), (2, 8)])
+def test_symmetric_quantizers_other_widths_bit_exact(tlq, w_bits, a_bits):
+    xb = wl.activations(71, "sym/x", 130, 1040, 96, "normal", 4)
+    wb = wl.weights(71, "sym/w", 77, 1040)
+    s_np = orc.scale_table(orc.channel_stat(xb), 20)[9]
+    cfg = tlq.config(tlq.WA_SYM_CHANNEL, w_bits=w_bits, a_bits=a_bits)
+    for s_vec in (None, s_np):
+        s_dev = None if s_vec is None else dev_bf16(tlq, orc.f32_to_bf16_bits(s_vec))
+        out = tlq.tlq_quantize_weights(dev_bf16(tlq, wb), s_dev, cfg)
+        codes, steps = tlq.tlq_quantize_activations(dev_bf16(tlq, xb), s_dev, cfg)
+        torch.cuda.synchronize()
+        qw, u = orc.quantize_weights_row_sym(wb, s_vec, w_bits)
+        qx, t = orc.quantize_activations_token_sym(xb, s_vec, a_bits)
+        assert np.array_equal(out["codes"].cpu().numpy(), qw)
+        assert np.array_equal(out["steps"].cpu().numpy().view(np.uint32), u.view(np.uint32))
+        assert np.array_equal(codes.cpu().numpy(), qx)
+        assert np.array_equal(steps.cpu().numpy().view(np.uint32), t.view(np.uint32))
+        assert qw.min() >= -(1 << (w_bits - 1)) and qx.max() <= (1 << (a_bits - 1)) - 1
+
+
+def run_search_sym(tlq, xb, wb, imp, w_bits, a_bits, n_grid=20):
+    cfg = tlq.config(tlq.WA_SYM_CHANNEL, w_bits=w_bits, a_bits=a_bits, n_grid=n_grid)
+    w_dev = None if imp is None else torch.from_numpy(np.asarray(imp, dtype=np.float32)).cuda()
+    out = tlq.tlq_scale_search_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), w_dev, cfg, per_token=True)
+    return dict(best=int(out.best_idx.item()), losses=out.losses.cpu().numpy(), per_token=out.per_token.cpu().numpy(),
+                s_best=bits_of(out.s_best))
+
+
+@pytest.mark.parametrize("mode,n,c1,c2,n_grid", [("w4a8", 256, 512, 512, 20), ("w4a6", 256, 512, 512, 20),
+                                                 ("w4a8", 515, 1088, 777, 6), ("w4a6", 300, 208, 320, 5)])
+def test_search_w4a8_w4a6(tlq, mode, n, c1, c2, n_grid):
+    xb, wb, imp = wl.small_case(73, n, c1, c2, n_outlier=2)
+    wn, an = orc.symmetric_bits(mode)
+    ref = orc.scale_search(xb, wb, imp, mode, 0, n_grid)
+    got = run_search_sym(tlq, xb, wb, imp, wn, an, n_grid)
+    check_against_oracle(got, ref, n_grid)
+
+
+def test_apply_layer_w4a8(tlq):
+    xb, wb, imp = wl.small_case(79, 300, 256, 328)
+    ref = orc.scale_search(xb, wb, imp, "w4a8", 0, 8)
+    s = ref["scales"][ref["best"]]
+    yq_ref, (qw, u, _) = orc.apply_layer(xb, wb, s, None, "w4a8")
+    out = tlq.tlq_apply_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), dev_bf16(tlq, orc.f32_to_bf16_bits(s)), None,
+                              tlq.config(tlq.WA_SYM_CHANNEL, w_bits=4, a_bits=8))
+    assert np.array_equal(out["codes"].cpu().numpy(), qw)
+    assert np.array_equal(out["steps"].cpu().numpy().view(np.uint32), u.view(np.uint32))
+    yq = out["Yq"].float().cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(yq - yq_ref) <= 2.0 ** -8 * np.abs(yq_ref) + 1e-6)

@@ -294,7 +294,7 @@ def test_first_candidate_is_plain_rtn():
     assert np.array_equal(orc.candidate_error(x, w, None, "w8a8", 0), res8["per_token"][0])
 
 
-@pytest.mark.parametrize("mode", ["w4a16", "w8a8"])
+@pytest.mark.parametrize("mode", ["w4a16", "w8a8", "w4a8", "w4a6"])
 def test_search_agrees_with_scalar_brute_force(mode):
     x, w, imp = wl.small_case(51, 5, 8, 3)
     res = orc.scale_search(x, w, imp, mode=mode, group=4, n_grid=4, w_bits_n=3 if mode == "w4a16" else 4)
@@ -318,6 +318,31 @@ def test_w8a8_error_matches_explicit_dequantization():
     assert np.allclose(e, (d ** 2).sum(axis=1), rtol=1e-10)
     # 8-bit error is far below 4-bit group error on the same data
     assert e.sum() < 0.05 * orc.candidate_error(x, w, s, "w4a16", 64).sum()
+
+
+def test_paper_bit_widths_w4a8_w4a6():
+    """The paper's own settings (Experiments: W4A8 and W4A6, per-token symmetric activations, per-channel
+    symmetric weights): integer ranges follow [-2^(n-1), 2^(n-1)-1], the largest element of a row sits on
+    +-(2^(n-1)-1), and fewer bits can only cost accuracy on the same data."""
+    x, w, imp = wl.small_case(67, 32, 64, 12)
+    s = orc.scale_table(orc.channel_stat(x), 20)[10]
+    assert orc.symmetric_bits("w4a8") == (4, 8) and orc.symmetric_bits("w4a6") == (4, 6)
+    qw, u = orc.quantize_weights_row_sym(w, s, 4)
+    assert qw.min() >= -8 and qw.max() <= 7 and np.all(np.abs(qw).max(axis=1) == 7)
+    qx, t = orc.quantize_activations_token_sym(x, s, 6)
+    assert qx.min() >= -32 and qx.max() <= 31 and np.all(np.abs(qx).max(axis=1) == 31)
+    p = (orc.bf16_to_f64(w) * s[None, :].astype(np.float64))
+    assert np.allclose(u, np.abs(p).max(axis=1) / 7.0, rtol=1e-6)
+    e88 = orc.candidate_error(x, w, s, "w8a8", 0).sum()
+    e48 = orc.candidate_error(x, w, s, "w4a8", 0).sum()
+    e46 = orc.candidate_error(x, w, s, "w4a6", 0).sum()
+    assert e88 < e48 < e46
+    # the error of W4A8 is dominated by the 4-bit weights: explicit dequantization gives the same number
+    qx8, t8 = orc.quantize_activations_token_sym(x, s, 8)
+    d = orc.bf16_to_f64(x) @ orc.bf16_to_f64(w).T - (qx8 * t8[:, None].astype(np.float64)) @ (qw * u[:, None].astype(np.float64)).T
+    assert np.allclose(orc.candidate_error(x, w, s, "w4a8", 0), (d ** 2).sum(axis=1), rtol=1e-10)
+    with pytest.raises(ValueError):
+        orc.symmetric_bits("w9a8")
 
 
 def test_argmin_takes_lowest_index_on_ties():
