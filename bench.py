@@ -314,8 +314,8 @@ def run_ours(args, cfgw):
     achieved = gemm_flops_sum / (gemm_ms_sum * 1e-3) / 1e12 if gemm_ms_sum > 0 else None
     traffic = None
     tpath = os.path.join(ROOT, "profiles", "search_gemm_traffic.json")
-    if os.path.exists(tpath):
-        with open(tpath) as f:
+    if os.path.exists(tpath) and args.linears is None and args.mode is None:
+        with open(tpath) as f:      # ncu counters of this very workload and kernel; anything else has none
             traffic = json.load(f).get(cfgr.key)
     i8 = cfgr.mode != "w4a16"
     # int8 runs at twice the bf16 rate on these tensor cores (nominal 4500 vs 2250 dense): the int8 peak
