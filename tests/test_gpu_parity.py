@@ -360,3 +360,35 @@ def test_apply_layer_w4a8(tlq):
     assert np.array_equal(out["steps"].cpu().numpy().view(np.uint32), u.view(np.uint32))
     yq = out["Yq"].float().cpu().numpy().astype(np.float64)
     assert np.all(np.abs(yq - yq_ref) <= 2.0 ** -8 * np.abs(yq_ref) + 1e-6)
+
+
+# ----------------------------------------------------------------------------------- host-side pipeline
+
+
+def test_host_layer_search_overlapped_copies_match_direct_calls(tlq):
+    """Inputs in pinned host memory, copies on a side stream: same argmin and bit-identical losses as the direct
+    call on resident tensors, also when the staging buffers are re-used for new data right away."""
+    from paper_2602_07899_b200 import calibrate
+    dev = torch.device("cuda", 0)
+    cfg = tlq.config(n_grid=6)
+    shapes = [("a", "x0", 300, 256, 320), ("b", "x0", 300, 256, 64), ("c", "x1", 300, 512, 256)]
+    pipe = calibrate.HostLayerSearch(shapes, cfg, dev)
+    rounds = []
+    for seed in (81, 82, 83):
+        hx, hw = {}, {}
+        for name, x_name, n, c1, c2 in shapes:
+            xb, wb, imp = wl.small_case(seed + c1, n, c1, c2)
+            hx.setdefault(x_name, torch.from_numpy(xb.view(np.int16)).pin_memory())
+            hw[name] = torch.from_numpy(wb.view(np.int16)).pin_memory()
+        himp = torch.from_numpy(wl.importance(seed, "pipe/imp", 300, 225)).pin_memory()
+        out = {name: (torch.empty(1, dtype=torch.int32).pin_memory(), torch.empty(6, dtype=torch.float64).pin_memory())
+               for name, *_ in shapes}
+        pipe.run(hx, hw, himp, out)       # three rounds back to back, no host synchronisation in between
+        rounds.append((hx, hw, himp, out))
+    pipe.check()
+    for hx, hw, himp, out in rounds:
+        for name, x_name, n, c1, c2 in shapes:
+            ref = tlq.tlq_scale_search_layer(hx[x_name].cuda().view(torch.bfloat16), hw[name].cuda().view(torch.bfloat16),
+                                             himp.cuda(), cfg)
+            assert int(out[name][0].item()) == int(ref.best_idx.item())
+            assert np.array_equal(out[name][1].numpy().view(np.uint64), ref.losses.cpu().numpy().view(np.uint64))
