@@ -64,6 +64,15 @@ extern "C" {
 #define TLQ_DTYPE_BF16 0
 #define TLQ_DTYPE_F32 1
 
+/* tlq_config.flags */
+#define TLQ_FLAG_SKIP_ZERO_WEIGHT_TOKENS 1u /* tlq_scale_search_layer: tokens whose importance weight is not > 0 add
+                                               nothing to any loss, so the quantized layer is applied only to the
+                                               others (packed on the device, order kept).  With the paper's Top-50%
+                                               token set as a 0/1 weight vector (Sec. 3.1.2) this halves the tensor
+                                               work.  x_stat still sees every token (or those of `mask`).  Needs
+                                               w_imp; per_token_err must be NULL.  Losses equal the unflagged call's
+                                               up to the order of the fp32 partial sums. */
+
 #define TLQ_MAX_GRID 64
 
 typedef struct {
@@ -74,7 +83,7 @@ typedef struct {
   int32_t group_size;   /* 32, 64, 128 or 256 for the group mode (must divide C1); ignored for W8A8 */
   int32_t n_grid;       /* K >= 1; candidate k uses r_k = k / K, so candidate 0 is scale = 1 */
   int32_t stat_mode;    /* TLQ_STAT_* */
-  uint32_t flags;       /* reserved, must be 0 */
+  uint32_t flags;       /* TLQ_FLAG_* bits, 0 by default */
 } tlq_config;
 
 /* Stages of tlq_scale_search_layer, for tlq_stage_timing_drain(). */

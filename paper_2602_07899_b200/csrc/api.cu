@@ -15,7 +15,7 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 int check_cfg(const tlq_config* cfg, int64_t C1, bool need_quantizer = true) {
   if (cfg == nullptr || cfg->struct_size != sizeof(tlq_config)) return TLQ_ERR_INVALID_ARG;
-  if (cfg->flags != 0) return TLQ_ERR_INVALID_ARG;
+  if ((cfg->flags & ~(uint32_t)TLQ_FLAG_SKIP_ZERO_WEIGHT_TOKENS) != 0) return TLQ_ERR_INVALID_ARG;
   if (cfg->n_grid < 1 || cfg->n_grid > TLQ_MAX_GRID) return TLQ_ERR_SHAPE;
   if (cfg->stat_mode < TLQ_STAT_MEAN_ABS || cfg->stat_mode > TLQ_STAT_MASKED_MAX) return TLQ_ERR_INVALID_ARG;
   if (C1 < 8 || (C1 % 8) != 0) return TLQ_ERR_SHAPE;
@@ -70,6 +70,10 @@ struct SearchLayout {
   float* u;
   int8_t* Xq;
   float* t;
+  int32_t* live;         // token compaction: live[0] = live tokens, live[1] = rounded up to 128
+  int32_t* live_idx;     // [N] source row of each packed row
+  float* wc;             // [n_pad] packed weights
+  uint16_t* Xc;          // [n_pad, C1] packed activations
   size_t bytes;
   GemmPlan plan;
   int64_t ptab_slices;   // per-candidate slices of the per-token table (column tiles, x2 for W8A8)
@@ -96,6 +100,12 @@ SearchLayout carve_search(void* ws, int64_t N, int64_t C1, int64_t C2, const tlq
     L.u = c.take<float>((size_t)K * C2);
     L.Xq = c.take<int8_t>((size_t)K * N * C1, 1024);
     L.t = c.take<float>((size_t)K * N);
+  }
+  if (cfg->flags & TLQ_FLAG_SKIP_ZERO_WEIGHT_TOKENS) {
+    L.live = c.take<int32_t>(2);
+    L.live_idx = c.take<int32_t>((size_t)N);
+    L.wc = c.take<float>((size_t)L.plan.n_pad);
+    L.Xc = c.take<uint16_t>((size_t)L.plan.n_pad * C1, 1024);
   }
   L.bytes = align_up(c.off, 256);
   return L;
@@ -246,7 +256,7 @@ int tlq_quantize_activations(const void* X, const void* s, int64_t N, int64_t C1
   rc = have_device();
   if (rc != TLQ_OK) return rc;
   return launch_actquant_i8(reinterpret_cast<const uint16_t*>(X), reinterpret_cast<const uint16_t*>(s), nullptr, 1, N,
-                            C1, cfg->a_bits, codes, steps, reinterpret_cast<cudaStream_t>(stream));
+                            C1, cfg->a_bits, codes, steps, nullptr, reinterpret_cast<cudaStream_t>(stream));
 }
 
 size_t tlq_scale_search_workspace_bytes(int64_t N, int64_t C1, int64_t C2, const tlq_config* cfg) {
@@ -263,6 +273,9 @@ int tlq_scale_search_layer(const void* X, int64_t N, int64_t C1, const void* W, 
   int rc = check_cfg(cfg, C1);
   if (rc != TLQ_OK) return rc;
   if (cfg->stat_mode == TLQ_STAT_MASKED_MAX && mask == nullptr) return TLQ_ERR_INVALID_ARG;
+  // skipping needs weights to look at; per-token errors of skipped tokens would not exist
+  const bool compact = (cfg->flags & TLQ_FLAG_SKIP_ZERO_WEIGHT_TOKENS) != 0;
+  if (compact && (w_imp == nullptr || per_token_err != nullptr)) return TLQ_ERR_INVALID_ARG;
   if (!aligned16(X) || !aligned16(W) || !aligned16(workspace)) return TLQ_ERR_ALIGN;
   SearchLayout L = carve_search(workspace, N, C1, C2, cfg);
   if (workspace_bytes < L.bytes) return TLQ_ERR_WORKSPACE;
@@ -281,17 +294,27 @@ int tlq_scale_search_layer(const void* X, int64_t N, int64_t C1, const void* W, 
     return rc;
   if ((rc = timing_mark(1, st)) != TLQ_OK) return rc;
   float* ptab = (per_token_err != nullptr) ? L.ptab : nullptr;
+  // tokens of zero weight cannot change any loss: pack the others to the front and run the layer on those only
+  const uint16_t* Xg = Xb;          // what the quantized layer is applied to
+  const float* wg = w_imp;
+  const int32_t* n_live = nullptr;
+  if (compact) {
+    if ((rc = launch_compact_tokens(Xb, w_imp, N, L.plan.n_pad, C1, L.live_idx, L.wc, L.live, L.Xc, st)) != TLQ_OK)
+      return rc;
+    TLQ_CUDA_TRY(cudaMemsetAsync(L.partials, 0, (size_t)K * L.plan.partials_per_k * sizeof(float), st));
+    Xg = L.Xc; wg = L.wc; n_live = L.live;
+  }
   if (cfg->mode == TLQ_W4A16_ASYM_GROUP) {
     if ((rc = launch_fakequant_group(Wb, L.s, L.rs, K, C2, C1, cfg->group_size, cfg->w_bits, L.dW, nullptr, nullptr,
                                      nullptr, st)) != TLQ_OK)
       return rc;
     if ((rc = timing_mark(2, st)) != TLQ_OK) return rc;
-    if ((rc = launch_search_gemm_bf16(Xb, L.dW, w_imp, L.plan, L.partials, ptab, L.hdr, st)) != TLQ_OK) return rc;
+    if ((rc = launch_search_gemm_bf16(Xg, L.dW, wg, L.plan, L.partials, ptab, L.hdr, n_live, st)) != TLQ_OK) return rc;
   } else {
     if ((rc = launch_fakequant_rows_i8(Wb, L.s, K, C2, C1, cfg->w_bits, L.Wq, L.u, st)) != TLQ_OK) return rc;
-    if ((rc = launch_actquant_i8(Xb, nullptr, L.rs, K, N, C1, cfg->a_bits, L.Xq, L.t, st)) != TLQ_OK) return rc;
+    if ((rc = launch_actquant_i8(Xg, nullptr, L.rs, K, N, C1, cfg->a_bits, L.Xq, L.t, n_live, st)) != TLQ_OK) return rc;
     if ((rc = timing_mark(2, st)) != TLQ_OK) return rc;
-    if ((rc = launch_search_gemm_i8(Xb, Wb, L.Xq, L.Wq, L.t, L.u, w_imp, L.plan, L.partials, ptab, L.hdr, st)) !=
+    if ((rc = launch_search_gemm_i8(Xg, Wb, L.Xq, L.Wq, L.t, L.u, wg, L.plan, L.partials, ptab, L.hdr, n_live, st)) !=
         TLQ_OK)
       return rc;
   }
@@ -364,7 +387,7 @@ int tlq_apply_layer(const void* X, int64_t N, int64_t C1, const void* W, int64_t
     return launch_apply_gemm_bf16(Xb, Wb, L.dW, bb, N, C1, C2, reinterpret_cast<uint16_t*>(Yq), L.hdr, st);
   }
   if ((rc = launch_fakequant_rows_i8(Wb, sb, 1, C2, C1, cfg->w_bits, L.Wq, L.u, st)) != TLQ_OK) return rc;
-  if ((rc = launch_actquant_i8(Xb, sb, nullptr, 1, N, C1, cfg->a_bits, L.Xq, L.t, st)) != TLQ_OK) return rc;
+  if ((rc = launch_actquant_i8(Xb, sb, nullptr, 1, N, C1, cfg->a_bits, L.Xq, L.t, nullptr, st)) != TLQ_OK) return rc;
   if (codes != nullptr) TLQ_CUDA_TRY(cudaMemcpyAsync(codes, L.Wq, (size_t)C2 * C1, cudaMemcpyDeviceToDevice, st));
   if (steps != nullptr) TLQ_CUDA_TRY(cudaMemcpyAsync(steps, L.u, (size_t)C2 * sizeof(float), cudaMemcpyDeviceToDevice, st));
   return launch_apply_gemm_i8(L.Xq, L.Wq, L.t, L.u, bb, N, C1, C2, reinterpret_cast<uint16_t*>(Yq), L.hdr, st);

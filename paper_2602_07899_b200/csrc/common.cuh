@@ -133,8 +133,14 @@ int launch_fakequant_group(const uint16_t* W, const uint16_t* s /*[K,C1] or null
 int launch_fakequant_rows_i8(const uint16_t* W, const uint16_t* s /*[K,C1] or null*/, int K, int64_t C2, int64_t C1,
                              int bits, int8_t* q /*[K,C2,C1]*/, float* u /*[K,C2]*/, cudaStream_t st);
 // activations: x * (1/s); give the reciprocal table rs [K,C1], or a bf16 scale s [K,C1] to invert on the fly, or neither
+// n_rows_dev: optional device int32 holding how many leading rows are live (the rest are skipped)
 int launch_actquant_i8(const uint16_t* X, const uint16_t* s, const float* rs, int K, int64_t N, int64_t C1, int bits,
-                       int8_t* q /*[K,N,C1]*/, float* t /*[K,N]*/, cudaStream_t st);
+                       int8_t* q /*[K,N,C1]*/, float* t /*[K,N]*/, const int32_t* n_rows_dev, cudaStream_t st);
+
+// compact.cu: pack the rows of X whose weight is > 0 to the front (order kept); live[0] = count, live[1] = count
+// rounded up to 128.  idx [N], wc [n_pad], Xc [n_pad, C1].
+int launch_compact_tokens(const uint16_t* X, const float* w_imp, int64_t N, int64_t n_pad, int64_t C1, int32_t* idx,
+                          float* wc, int32_t* live, uint16_t* Xc, cudaStream_t st);
 
 // importance.cu
 int launch_token_importance(const void* G, int g_dtype, int64_t B, int64_t N, int64_t C, int norm_kind,
@@ -158,8 +164,9 @@ struct GemmPlan {
 };
 GemmPlan plan_search_gemm(int64_t N, int64_t C1, int64_t C2, int K);
 // W4A16 search: partials[K][mtiles*otiles*4] (+ ptab[K][otiles][n_pad] if non-null)
+// n_live: optional device int32: only the first *n_live rows of X are tokens (the partial buffer must be zeroed)
 int launch_search_gemm_bf16(const uint16_t* X, const uint16_t* dW, const float* w_imp, const GemmPlan& plan,
-                            float* partials, float* ptab, WorkspaceHeader* hdr, cudaStream_t st);
+                            float* partials, float* ptab, WorkspaceHeader* hdr, const int32_t* n_live, cudaStream_t st);
 // Apply: Yq[N,C2] = X W^T - X dW^T (+bias), bf16 out
 int launch_apply_gemm_bf16(const uint16_t* X, const uint16_t* W, const uint16_t* dW, const uint16_t* bias,
                            int64_t N, int64_t C1, int64_t C2, uint16_t* Yq, WorkspaceHeader* hdr, cudaStream_t st);
@@ -169,7 +176,7 @@ GemmPlan plan_search_gemm_i8(int64_t N, int64_t C1, int64_t C2, int K);   // par
 // W8A8 search: partials[K][mtiles*otiles*8] (+ ptab[K][otiles*2][n_pad] if non-null)
 int launch_search_gemm_i8(const uint16_t* X, const uint16_t* W, const int8_t* Xq, const int8_t* Wq, const float* t,
                           const float* u, const float* w_imp, const GemmPlan& plan, float* partials, float* ptab,
-                          WorkspaceHeader* hdr, cudaStream_t st);
+                          WorkspaceHeader* hdr, const int32_t* n_live, cudaStream_t st);
 // Apply: Yq[N,C2] = t[n] * u[o] * (Xq Wq^T) (+bias), bf16 out
 int launch_apply_gemm_i8(const int8_t* Xq, const int8_t* Wq, const float* t, const float* u, const uint16_t* bias,
                          int64_t N, int64_t C1, int64_t C2, uint16_t* Yq, WorkspaceHeader* hdr, cudaStream_t st);

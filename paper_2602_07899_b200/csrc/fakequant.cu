@@ -486,11 +486,14 @@ __device__ __forceinline__ void unpack16(const uint4& t0, const uint4& t1, float
 template <int kKind>
 __global__ void __launch_bounds__(kGqThreads, 3)
 row_amax_kernel(const uint16_t* __restrict__ src, const uint16_t* __restrict__ s_tab, const float* __restrict__ rs_tab,
-                int K, int k_per_cta, int64_t R, int64_t C1, int* __restrict__ amax_bits /*[K,R], zeroed*/) {
+                int K, int k_per_cta, int64_t R_all, const int32_t* __restrict__ n_rows_dev, int64_t C1,
+                int* __restrict__ amax_bits /*[K,R_all], zeroed*/) {
   __shared__ uint4 tile[kGqRows][kGqCols / 8];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t c0 = (int64_t)blockIdx.x * kGqCols + lane * 16;
   const int64_t row0 = (int64_t)blockIdx.y * kGqRows;
+  const int64_t R = (n_rows_dev != nullptr) ? (int64_t)*n_rows_dev : R_all;    // rows beyond are not live
+  if (row0 >= R) return;                                                        // the whole CTA leaves together
   const bool col_ok = c0 < C1;
   stage_tile(tile, src, row0, R, C1, c0, col_ok, warp, lane);
   const int k_begin = blockIdx.z * k_per_cta;
@@ -513,7 +516,7 @@ row_amax_kernel(const uint16_t* __restrict__ src, const uint16_t* __restrict__ s
       }
 #pragma unroll
       for (int off = 16; off > 0; off >>= 1) a = fmaxf(a, __shfl_xor_sync(0xFFFFFFFFu, a, off));
-      if (lane == 0) atomicMax(amax_bits + (int64_t)k * R + row0 + r, __float_as_int(a));
+      if (lane == 0) atomicMax(amax_bits + (int64_t)k * R_all + row0 + r, __float_as_int(a));
     }
   }
 }
@@ -544,12 +547,15 @@ __device__ __noinline__ void codes16_exact(const uint4* tile16, const float* mul
 template <int kKind>
 __global__ void __launch_bounds__(kGqThreads, 3)
 row_codes_kernel(const uint16_t* __restrict__ src, const uint16_t* __restrict__ s_tab, const float* __restrict__ rs_tab,
-                 const float* __restrict__ step /*[K,R]*/, int K, int k_per_cta, int64_t R, int64_t C1, float qpos,
-                 float tie_eps, int8_t* __restrict__ q /*[K,R,C1]*/) {
+                 const float* __restrict__ step /*[K,R_all]*/, int K, int k_per_cta, int64_t R_all,
+                 const int32_t* __restrict__ n_rows_dev, int64_t C1, float qpos, float tie_eps,
+                 int8_t* __restrict__ q /*[K,R_all,C1]*/) {
   __shared__ uint4 tile[kGqRows][kGqCols / 8];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t c0 = (int64_t)blockIdx.x * kGqCols + lane * 16;
   const int64_t row0 = (int64_t)blockIdx.y * kGqRows;
+  const int64_t R = (n_rows_dev != nullptr) ? (int64_t)*n_rows_dev : R_all;
+  if (row0 >= R) return;
   const bool col_ok = c0 < C1;
   stage_tile(tile, src, row0, R, C1, c0, col_ok, warp, lane);
   if (!col_ok) return;                    // no warp-wide operation below
@@ -566,7 +572,7 @@ row_codes_kernel(const uint16_t* __restrict__ src, const uint16_t* __restrict__ 
       const int r = p * 8 + warp;
       const int64_t row = row0 + r;
       if (row >= R) break;
-      const float st = step[(int64_t)k * R + row];
+      const float st = step[(int64_t)k * R_all + row];
       const float inv = rcp_fast(st);
       const float2 inv2 = make_float2(inv, inv);
       float2 w[8];
@@ -582,7 +588,7 @@ row_codes_kernel(const uint16_t* __restrict__ src, const uint16_t* __restrict__ 
         tb[2 * j] = __float_as_uint(t.x);
         tb[2 * j + 1] = __float_as_uint(t.y);
       }
-      uint4* dst = reinterpret_cast<uint4*>(q + ((int64_t)k * R + row) * C1 + c0);
+      uint4* dst = reinterpret_cast<uint4*>(q + ((int64_t)k * R_all + row) * C1 + c0);
       if (near > tie_lim) {
         float mf[16];
 #pragma unroll
@@ -602,7 +608,7 @@ row_codes_kernel(const uint16_t* __restrict__ src, const uint16_t* __restrict__ 
 
 template <int kKind>
 static int launch_rows(const uint16_t* src, const uint16_t* s, const float* rs, int K, int64_t R, int64_t C1, int bits,
-                       int8_t* q, float* step, cudaStream_t st) {
+                       int8_t* q, float* step, const int32_t* n_rows_dev, cudaStream_t st) {
   const int64_t ctas = ceil_div(C1, kGqCols) * ceil_div(R, kGqRows);
   int64_t kchunks = ceil_div(148 * 6, ctas);
   if (kchunks > K) kchunks = K;
@@ -614,24 +620,25 @@ static int launch_rows(const uint16_t* src, const uint16_t* s, const float* rs, 
   const float tie_eps = 4.0e-7f * (qpos + 1.0f);
   const int64_t n = (int64_t)K * R;
   TLQ_CUDA_TRY(cudaMemsetAsync(step, 0, (size_t)n * sizeof(float), st));
-  row_amax_kernel<kKind><<<grid, kGqThreads, 0, st>>>(src, s, rs, K, k_per_cta, R, C1, reinterpret_cast<int*>(step));
+  row_amax_kernel<kKind><<<grid, kGqThreads, 0, st>>>(src, s, rs, K, k_per_cta, R, n_rows_dev, C1,
+                                                      reinterpret_cast<int*>(step));
   int rc = after_launch();
   if (rc != TLQ_OK) return rc;
   amax_to_step_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(step, n, qpos);
   if ((rc = after_launch()) != TLQ_OK) return rc;
-  row_codes_kernel<kKind><<<grid, kGqThreads, 0, st>>>(src, s, rs, step, K, k_per_cta, R, C1, qpos, tie_eps, q);
+  row_codes_kernel<kKind><<<grid, kGqThreads, 0, st>>>(src, s, rs, step, K, k_per_cta, R, n_rows_dev, C1, qpos, tie_eps, q);
   return after_launch();
 }
 
 int launch_fakequant_rows_i8(const uint16_t* W, const uint16_t* s, int K, int64_t C2, int64_t C1, int bits, int8_t* q,
                              float* u, cudaStream_t st) {
-  return launch_rows<kMultScale>(W, s, nullptr, K, C2, C1, bits, q, u, st);
+  return launch_rows<kMultScale>(W, s, nullptr, K, C2, C1, bits, q, u, nullptr, st);
 }
 
 int launch_actquant_i8(const uint16_t* X, const uint16_t* s, const float* rs, int K, int64_t N, int64_t C1, int bits,
-                       int8_t* q, float* t, cudaStream_t st) {
-  if (rs != nullptr) return launch_rows<kMultRecipTable>(X, nullptr, rs, K, N, C1, bits, q, t, st);
-  return launch_rows<kMultRecipOfScale>(X, s, nullptr, K, N, C1, bits, q, t, st);
+                       int8_t* q, float* t, const int32_t* n_rows_dev, cudaStream_t st) {
+  if (rs != nullptr) return launch_rows<kMultRecipTable>(X, nullptr, rs, K, N, C1, bits, q, t, n_rows_dev, st);
+  return launch_rows<kMultRecipOfScale>(X, s, nullptr, K, N, C1, bits, q, t, n_rows_dev, st);
 }
 
 }  // namespace tlq

@@ -44,6 +44,7 @@ struct GemmArgs {
   int64_t num_tiles;       // K * otiles * mtiles
   int64_t tiles_per_k;     // otiles * mtiles
   TileRaster raster;       // walk order inside one candidate
+  const int32_t* n_live;   // device: live token count after compaction, or null (= N)
   int64_t n_pad;
   const float* w_imp;      // [N] or null (uniform)
   float* partials;         // [K][otiles*mtiles*4]
@@ -98,6 +99,17 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
   const int passes = kApply ? 2 : 1;
   const int num_kb = args.num_kb;
+  // token count and tile walk: fixed by the host, or read from the device when the tokens were compacted
+  int64_t n_tokens = args.N, tiles_per_k = args.tiles_per_k, num_tiles = args.num_tiles;
+  TileRaster raster = args.raster;
+  if (args.n_live != nullptr) {
+    n_tokens = *args.n_live;
+    const int64_t mt_live = (n_tokens + BM - 1) / BM;
+    raster.mtiles = (int)mt_live;
+    if (raster.b == 1) raster.a = mt_live > 0 ? (int)mt_live : 1;
+    tiles_per_k = args.otiles * mt_live;
+    num_tiles = (args.num_tiles / args.tiles_per_k) * tiles_per_k;
+  }
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -105,10 +117,10 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int64_t tile = blockIdx.x; tile < args.num_tiles && ok; tile += gridDim.x) {
-        const int k = (int)(tile / args.tiles_per_k);
+      for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        const int k = (int)(tile / tiles_per_k);
         int mt, ot;
-        args.raster.decode(tile - (int64_t)k * args.tiles_per_k, mt, ot);
+        raster.decode(tile - (int64_t)k * tiles_per_k, mt, ot);
         for (int pass = 0; pass < passes && ok; ++pass) {
           const CUtensorMap* tb = (kApply && pass == 1) ? &tmB2 : &tmB;
           for (int kb = 0; kb < num_kb; ++kb) {
@@ -133,7 +145,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       uint32_t phase = 0;
       int64_t it = 0;
       bool ok = true;
-      for (int64_t tile = blockIdx.x; tile < args.num_tiles && ok; tile += gridDim.x, ++it) {
+      for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
         const int acc = (int)(it & 1);
         const uint32_t acc_phase = (uint32_t)((it >> 1) & 1);
         if (!ptx::mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) {
@@ -173,10 +185,10 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int quarter = warp & 3;                 // tensor-memory lanes [32*quarter, 32*quarter+32)
     const int row_in_tile = quarter * 32 + lane;
     int64_t it = 0;
-    for (int64_t tile = blockIdx.x; tile < args.num_tiles; tile += gridDim.x, ++it) {
-      const int k = (int)(tile / args.tiles_per_k);
+    for (int64_t tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
+      const int k = (int)(tile / tiles_per_k);
       int mt, ot;
-      args.raster.decode(tile - (int64_t)k * args.tiles_per_k, mt, ot);
+      raster.decode(tile - (int64_t)k * tiles_per_k, mt, ot);
       const int acc = (int)(it & 1);
       const uint32_t acc_phase = (uint32_t)((it >> 1) & 1);
       if (!ptx::mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) {
@@ -206,7 +218,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const float e = (s0 + s1) + (s2 + s3);      // sum_o E[n,o]^2 over this tile's 256 output channels
         if (args.ptab != nullptr) args.ptab[((int64_t)k * args.otiles + ot) * args.n_pad + n] = e;
         float wn = 0.0f;
-        if (n < args.N) wn = (args.w_imp != nullptr) ? args.w_imp[n] : 1.0f;
+        if (n < n_tokens) wn = (args.w_imp != nullptr) ? args.w_imp[n] : 1.0f;
         float v = wn * e;
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
@@ -219,7 +231,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           ptx::tmem_ld32(taddr + c * 32, r);
           ptx::tmem_ld_wait();
           const int64_t col0 = (int64_t)ot * BN + c * 32;
-          if (n < args.N) {
+          if (n < n_tokens) {
 #pragma unroll
             for (int p = 0; p < 4; ++p) {
               const int64_t col = col0 + p * 8;
@@ -327,7 +339,7 @@ static bool make_maps_bf16(const uint16_t* X, int64_t N, int64_t C1, const uint1
 }
 
 int launch_search_gemm_bf16(const uint16_t* X, const uint16_t* dW, const float* w_imp, const GemmPlan& plan,
-                            float* partials, float* ptab, WorkspaceHeader* hdr, cudaStream_t st) {
+                            float* partials, float* ptab, WorkspaceHeader* hdr, const int32_t* n_live, cudaStream_t st) {
   CUtensorMap tmA, tmB;
   if (!make_maps_bf16(X, plan.N, plan.C1, dW, plan.C2, plan.K, &tmA, &tmB)) return TLQ_ERR_CUDA;
   int rc = configure_kernel<false>();
@@ -340,6 +352,7 @@ int launch_search_gemm_bf16(const uint16_t* X, const uint16_t* dW, const float* 
   a.num_tiles = (int64_t)plan.K * a.tiles_per_k;
   a.n_pad = plan.n_pad;
   a.w_imp = w_imp; a.partials = partials; a.ptab = ptab; a.bias = nullptr; a.yq = nullptr; a.hdr = hdr;
+  a.n_live = n_live;
   const int sms = num_sms();
   if (sms <= 0) return TLQ_ERR_CUDA;
   const unsigned grid = (unsigned)(a.num_tiles < sms ? a.num_tiles : sms);

@@ -48,6 +48,7 @@ struct I8Args {
   int64_t mtiles, otiles;
   int64_t num_tiles;       // otiles * mtiles (every tile runs all passes)
   TileRaster raster;       // walk order of the tiles
+  const int32_t* n_live;   // device: live token count after compaction, or null (= N)
   int64_t n_pad;
   const float* w_imp;      // [N] or null
   const float* t;          // [K,N] activation steps
@@ -106,6 +107,16 @@ gemm_w8a8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
 
   // pass 0 of a search tile is the full-precision product; apply has the single int8 pass only
   const int passes = kApply ? 1 : args.K + 1;
+  // token count and tile walk: fixed by the host, or read from the device when the tokens were compacted
+  int64_t n_tokens = args.N, num_tiles = args.num_tiles;
+  TileRaster raster = args.raster;
+  if (args.n_live != nullptr) {
+    n_tokens = *args.n_live;
+    const int64_t mt_live = (n_tokens + BM - 1) / BM;
+    raster.mtiles = (int)mt_live;
+    if (raster.b == 1) raster.a = mt_live > 0 ? (int)mt_live : 1;
+    num_tiles = args.otiles * mt_live;
+  }
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -113,9 +124,9 @@ gemm_w8a8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int64_t tile = blockIdx.x; tile < args.num_tiles && ok; tile += gridDim.x) {
+      for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         int mt, ot;
-        args.raster.decode(tile, mt, ot);
+        raster.decode(tile, mt, ot);
         for (int pass = 0; pass < passes && ok; ++pass) {
           const bool fp = !kApply && pass == 0;
           const int k = kApply ? 0 : pass - 1;
@@ -147,7 +158,7 @@ gemm_w8a8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       uint32_t phase = 0;
       int64_t it = 0;                      // passes issued so far: selects the accumulator
       bool ok = true;
-      for (int64_t tile = blockIdx.x; tile < args.num_tiles && ok; tile += gridDim.x) {
+      for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         for (int pass = 0; pass < passes && ok; ++pass, ++it) {
           const bool fp = !kApply && pass == 0;
           const int nkb = fp ? args.num_kb16 : args.num_kb8;
@@ -194,9 +205,9 @@ gemm_w8a8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     float yfp[128];                               // this thread's share of the full-precision tile
     int64_t it = 0;
     bool ok = true;
-    for (int64_t tile = blockIdx.x; tile < args.num_tiles && ok; tile += gridDim.x) {
+    for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
       int mt, ot;
-      args.raster.decode(tile, mt, ot);
+      raster.decode(tile, mt, ot);
       const int64_t n = (int64_t)mt * BM + row_in_tile;
       const int64_t col_base = (int64_t)ot * BN + half * 128;
       for (int pass = 0; pass < passes; ++pass, ++it) {
@@ -224,7 +235,7 @@ gemm_w8a8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
           continue;
         }
         const int k = kApply ? 0 : pass - 1;
-        const float tn = (n < args.N) ? args.t[(int64_t)k * args.N + n] : 0.0f;
+        const float tn = (n < n_tokens) ? args.t[(int64_t)k * args.N + n] : 0.0f;
         const float* u_row = args.u + (int64_t)k * args.C2;
         if (!kApply) {
           float s0 = 0.f, s1 = 0.f;
@@ -253,7 +264,7 @@ gemm_w8a8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
           const float e = s0 + s1;                // sum over this warp's 128 output channels
           if (args.ptab != nullptr) args.ptab[((int64_t)k * args.otiles * 2 + ot * 2 + half) * args.n_pad + n] = e;
           float wn = 0.0f;
-          if (n < args.N) wn = (args.w_imp != nullptr) ? args.w_imp[n] : 1.0f;
+          if (n < n_tokens) wn = (args.w_imp != nullptr) ? args.w_imp[n] : 1.0f;
           float v = wn * e;
 #pragma unroll
           for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
@@ -265,7 +276,7 @@ gemm_w8a8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             uint32_t r[16];
             ptx::tmem_ld16(taddr + c * 16, r);
             ptx::tmem_ld_wait();
-            if (n < args.N) {
+            if (n < n_tokens) {
 #pragma unroll
               for (int p = 0; p < 2; ++p) {
                 const int64_t col = col_base + c * 16 + p * 8;
@@ -353,7 +364,7 @@ GemmPlan plan_search_gemm_i8(int64_t N, int64_t C1, int64_t C2, int K) {
 
 int launch_search_gemm_i8(const uint16_t* X, const uint16_t* W, const int8_t* Xq, const int8_t* Wq, const float* t,
                           const float* u, const float* w_imp, const GemmPlan& plan, float* partials, float* ptab,
-                          WorkspaceHeader* hdr, cudaStream_t st) {
+                          WorkspaceHeader* hdr, const int32_t* n_live, cudaStream_t st) {
   CUtensorMap tmX, tmW, tmXq, tmWq;
   if (!map_bf16_2d(&tmX, X, plan.N, plan.C1, BM) || !map_bf16_2d(&tmW, W, plan.C2, plan.C1, BN) ||
       !map_i8_3d(&tmXq, Xq, plan.N, plan.C1, plan.K, BM) || !map_i8_3d(&tmWq, Wq, plan.C2, plan.C1, plan.K, BN))
@@ -370,6 +381,7 @@ int launch_search_gemm_i8(const uint16_t* X, const uint16_t* W, const int8_t* Xq
   a.n_pad = plan.n_pad;
   a.w_imp = w_imp; a.t = t; a.u = u; a.partials = partials; a.ptab = ptab; a.bias = nullptr; a.yq = nullptr;
   a.hdr = hdr;
+  a.n_live = n_live;
   const int sms = sm_count();
   if (sms <= 0) return TLQ_ERR_CUDA;
   const unsigned grid = (unsigned)(a.num_tiles < sms ? a.num_tiles : sms);

@@ -47,13 +47,16 @@ class Config(ctypes.Structure):
                 ("stat_mode", ctypes.c_int32), ("flags", ctypes.c_uint32)]
 
 
+FLAG_SKIP_ZERO_WEIGHT_TOKENS = 1
+
+
 def config(mode: int = W4A16_ASYM_GROUP, w_bits: Optional[int] = None, a_bits: Optional[int] = None,
-           group_size: int = 128, n_grid: int = 20, stat_mode: int = STAT_MEAN_ABS) -> Config:
+           group_size: int = 128, n_grid: int = 20, stat_mode: int = STAT_MEAN_ABS, flags: int = 0) -> Config:
     if w_bits is None:
         w_bits = 4 if mode == W4A16_ASYM_GROUP else 8
     if a_bits is None:
         a_bits = 16 if mode == W4A16_ASYM_GROUP else 8
-    return Config(ctypes.sizeof(Config), mode, w_bits, a_bits, group_size, n_grid, stat_mode, 0)
+    return Config(ctypes.sizeof(Config), mode, w_bits, a_bits, group_size, n_grid, stat_mode, flags)
 
 
 def _load() -> ctypes.CDLL:

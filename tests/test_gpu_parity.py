@@ -392,3 +392,76 @@ def test_host_layer_search_overlapped_copies_match_direct_calls(tlq):
                                              himp.cuda(), cfg)
             assert int(out[name][0].item()) == int(ref.best_idx.item())
             assert np.array_equal(out[name][1].numpy().view(np.uint64), ref.losses.cpu().numpy().view(np.uint64))
+
+
+def test_shared_scale_search_on_stacked_sibling_weights(tlq):
+    """q/k/v-style siblings searched as one row-stacked matrix: parity with the oracle on the stack, and the
+    stack's per-token error is the sum of the siblings' (one scale for all of them)."""
+    xb, wq, imp = wl.small_case(93, 300, 256, 320)
+    _, wk, _ = wl.small_case(94, 300, 256, 72)
+    stack = np.concatenate([wq, wk], axis=0)
+    ref = orc.scale_search(xb, stack, imp, "w4a16", 64, 6)
+    got = run_search(tlq, xb, stack, imp, group=64, n_grid=6)
+    check_against_oracle(got, ref, 6)
+    parts = run_search(tlq, xb, wq, imp, group=64, n_grid=6)["per_token"] + run_search(tlq, xb, wk, imp, group=64, n_grid=6)["per_token"]
+    np.testing.assert_allclose(got["per_token"], parts, rtol=1e-5)
+
+
+# ----------------------------------------------------------------------------------- zero-weight tokens skipped
+
+
+def _search_losses(tlq, xb, wb, imp, cfg):
+    out = tlq.tlq_scale_search_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), torch.from_numpy(imp).cuda(), cfg)
+    return int(out.best_idx.item()), out.losses.cpu().numpy(), bits_of(out.s_best)
+
+
+@pytest.mark.parametrize("mode", ["w4a16", "w8a8", "w4a6"])
+@pytest.mark.parametrize("n,c1,c2,kind", [(300, 256, 320, "top50"), (515, 1088, 777, "sparse"), (256, 512, 512, "onehot"),
+                                          (384, 256, 256, "dense"), (130, 128, 64, "first_tile_only")])
+def test_search_skipping_zero_weight_tokens(tlq, mode, n, c1, c2, kind):
+    """The paper's token-level calibration set is a 0/1 weight vector (top half by gradient importance);
+    tokens of weight zero are packed away before the quantized layer is applied.  Same losses as the
+    oracle (which multiplies by the zeros) and as the unflagged call."""
+    xb, wb, imp = wl.small_case(97, n, c1, c2)
+    imp = imp.copy()
+    if kind == "top50":
+        gb = wl.token_gradients(97, "skip/g", 2, n, 64, (3 * n) // 4)
+        imp = orc.top_mask(orc.token_importance(gb)[0], 0.5).astype(np.float32)
+        assert imp.sum() == n // 2
+    elif kind == "sparse":
+        imp[np.random.default_rng(5).random(n) < 0.7] = 0.0
+    elif kind == "onehot":
+        imp = wl.importance(97, "skip/onehot", n, (3 * n) // 4, "onehot")
+    elif kind == "first_tile_only":
+        imp[100:] = 0.0
+    n_grid = 5
+    if mode == "w4a16":
+        base = dict(group_size=64, n_grid=n_grid)
+        ref = orc.scale_search(xb, wb, imp, "w4a16", 64, n_grid)
+    else:
+        wn, an = orc.symmetric_bits(mode)
+        base = dict(mode=tlq.WA_SYM_CHANNEL, w_bits=wn, a_bits=an, n_grid=n_grid)
+        ref = orc.scale_search(xb, wb, imp, mode, 0, n_grid)
+    best0, loss0, s0 = _search_losses(tlq, xb, wb, imp, tlq.config(**base))
+    best1, loss1, s1 = _search_losses(tlq, xb, wb, imp, tlq.config(flags=tlq.FLAG_SKIP_ZERO_WEIGHT_TOKENS, **base))
+    np.testing.assert_allclose(loss1, ref["losses"], rtol=LOSS_RTOL)
+    np.testing.assert_allclose(loss1, loss0, rtol=1e-5)
+    order = np.sort(ref["losses"])
+    if (order[1] - order[0]) / order[0] > 1e-5:
+        assert best1 == ref["best"] == best0
+    assert np.array_equal(s1, orc.f32_to_bf16_bits(ref["scales"][best1]))
+
+
+def test_skipping_needs_weights_and_has_no_per_token_table(tlq):
+    xb, wb, imp = wl.small_case(98, 64, 128, 64)
+    cfg = tlq.config(n_grid=3, flags=tlq.FLAG_SKIP_ZERO_WEIGHT_TOKENS)
+    with pytest.raises(tlq.TlqError) as e:
+        tlq.tlq_scale_search_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), None, cfg)
+    assert e.value.status == tlq.ERR_INVALID_ARG
+    with pytest.raises(tlq.TlqError) as e:
+        tlq.tlq_scale_search_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), torch.from_numpy(imp).cuda(), cfg, per_token=True)
+    assert e.value.status == tlq.ERR_INVALID_ARG
+    # every weight zero: no loss is defined, reported through the status word, not as a fault
+    with pytest.raises(tlq.TlqError) as e:
+        tlq.tlq_scale_search_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), torch.zeros(64).cuda(), cfg)
+    assert e.value.status == tlq.ERR_NONFINITE

@@ -398,3 +398,20 @@ def test_apply_layer_equals_search_candidate():
     yq, (codes, step, zero) = orc.apply_layer(x, w, s, bias, "w4a16", 128)
     e = orc.per_token_error(orc.layer_fp(x, w, orc.bf16_to_f64(bias)), yq)   # the bias cancels in the error
     assert np.allclose(e, res["per_token"][res["best"]], rtol=1e-9)
+
+
+def test_shared_scale_of_sibling_linears_is_the_search_on_stacked_rows():
+    """Linears fed by the same activations (q/k/v, gate/up) must share one scale, because the scale is folded
+    into the layer before them (Sec. 2.2, last sentence on fusing the smoothing factor).  Quantizers act per
+    output row (or per group inside a row), so stacking the weight matrices row-wise changes no code, and the
+    loss of the stack is the row-count-weighted mean of the single losses: per_token adds up."""
+    x, wq, imp = wl.small_case(91, 40, 64, 24)
+    _, wk, _ = wl.small_case(92, 40, 64, 8)
+    stack = np.concatenate([wq, wk], axis=0)
+    for mode, group in (("w4a16", 32), ("w4a8", 0)):
+        a = orc.scale_search(x, wq, imp, mode=mode, group=group, n_grid=5)
+        b = orc.scale_search(x, wk, imp, mode=mode, group=group, n_grid=5)
+        c = orc.scale_search(x, stack, imp, mode=mode, group=group, n_grid=5)
+        assert np.allclose(c["per_token"], a["per_token"] + b["per_token"], rtol=1e-12)
+        assert np.allclose(c["losses"], (24 * a["losses"] + 8 * b["losses"]) / 32, rtol=1e-12)
+        assert np.array_equal(c["scales"], a["scales"])
