@@ -181,11 +181,12 @@ def run_ours(args, cfgw):
     cfgr = dataclasses.replace(cfgw, seed=replicas.replica_seed(cfgw.seed, rank))
     data = wl.LayerData(cfgr)
     lins = [l for l in cfgr.linears() if args.linears is None or l.name in args.linears.split(",")]
+    flags = tlq.FLAG_SKIP_ZERO_WEIGHT_TOKENS if args.skip_zero_weight else 0
     if cfgr.mode == "w4a16":
-        cfg = tlq.config(mode=tlq.W4A16_ASYM_GROUP, group_size=cfgr.group, n_grid=cfgr.n_grid)
+        cfg = tlq.config(mode=tlq.W4A16_ASYM_GROUP, group_size=cfgr.group, n_grid=cfgr.n_grid, flags=flags)
     else:   # "w<n>a<m>": symmetric per-channel weights / per-token activations on the int8 tensor-core path
         wn, an = (int(v) for v in cfgr.mode[1:].split("a"))
-        cfg = tlq.config(mode=tlq.WA_SYM_CHANNEL, w_bits=wn, a_bits=an, n_grid=cfgr.n_grid)
+        cfg = tlq.config(mode=tlq.WA_SYM_CHANNEL, w_bits=wn, a_bits=an, n_grid=cfgr.n_grid, flags=flags)
 
     # host (pinned) copies for the end-to-end leg, device-resident copies for the kernel leg
     host_x, host_w, dev_x, dev_w = {}, {}, {}, {}
@@ -195,7 +196,10 @@ def run_ours(args, cfgw):
             dev_x[l.x_name] = host_x[l.x_name].to(dev, non_blocking=True).view(torch.bfloat16)
         host_w[l.name] = torch.from_numpy(data.w(l).view(np.int16)).pin_memory()
         dev_w[l.name] = host_w[l.name].to(dev, non_blocking=True).view(torch.bfloat16)
-    host_imp = torch.from_numpy(data.imp()).pin_memory()
+    imp_np = data.imp()
+    if args.importance == "top50":      # the paper's token set: 1 for the top half by importance, 0 for the rest
+        imp_np = (imp_np >= np.sort(imp_np)[len(imp_np) // 2]).astype(np.float32)
+    host_imp = torch.from_numpy(imp_np).pin_memory()
     dev_imp = host_imp.to(dev, non_blocking=True)
     ws_bytes = max(tlq.tlq_scale_search_workspace_bytes(cfgr.n_tokens, l.c_in, l.c_out, cfg) for l in lins)
     workspace = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
@@ -273,11 +277,12 @@ def run_ours(args, cfgw):
     # ---- roofline of the dominant kernel (the fused search GEMM), from the per-stage events of the timed region
     peaks = measured_peaks()
     per_linear = {}
+    live_frac = float((imp_np > 0).mean()) if args.skip_zero_weight else 1.0   # tokens the GEMM really processes
     gemm_ms_sum, gemm_flops_sum = 0.0, 0.0
     stage_tot = [0.0] * tlq.N_STAGES
     for i, rec in enumerate(stage_ms):
         l = lins[i % len(lins)]
-        fl = cfgr.flops_per_candidate(l) * cfgr.n_grid
+        fl = cfgr.flops_per_candidate(l) * cfgr.n_grid * live_frac
         d = per_linear.setdefault(l.name, {"gemm_ms": [], "flops": fl, "stages_ms": [0.0] * tlq.N_STAGES})
         d["gemm_ms"].append(rec[2])
         for j in range(tlq.N_STAGES):
@@ -307,7 +312,7 @@ def run_ours(args, cfgw):
     achieved = gemm_flops_sum / (gemm_ms_sum * 1e-3) / 1e12 if gemm_ms_sum > 0 else None
     traffic = None
     tpath = os.path.join(ROOT, "profiles", "search_gemm_traffic.json")
-    if os.path.exists(tpath) and args.linears is None and args.mode is None:
+    if os.path.exists(tpath) and args.linears is None and args.mode is None and not args.skip_zero_weight:
         with open(tpath) as f:      # ncu counters of this very workload and kernel; anything else has none
             traffic = json.load(f).get(cfgr.key)
     i8 = cfgr.mode != "w4a16"
@@ -340,7 +345,7 @@ def run_ours(args, cfgw):
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if cfgr.mode == "w4a16" else "int8", "data": "synthetic",
-            "config": {"workload": workload_name(cfgr) + ("" if args.linears is None else f" [subset: {args.linears}]"), "l2": "inputs_exceed_l2 (operands of one linear: 0.1-2.9 GB)",
+            "config": {"workload": workload_name(cfgr) + ("" if args.linears is None else f" [subset: {args.linears}]") + ("" if args.importance == "config" else f" [importance: {args.importance}]") + (" [zero-weight tokens skipped]" if args.skip_zero_weight else ""), "l2": "inputs_exceed_l2 (operands of one linear: 0.1-2.9 GB)",
                        "parallelism": f"replicas x{world} (one layer per rank, no collective)"},
             "gemm_tflops": achieved, "roofline": roofline, "cpu_baseline": cpu,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -359,6 +364,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="cfg1")
     ap.add_argument("--mode", default=None, help="override the config's setting: w4a16, w8a8, w4a8, w4a6")
+    ap.add_argument("--importance", default="config", choices=["config", "top50"],
+                    help="token weights: the config's (log-normal) or a 0/1 top-50%% mask (the paper's token set)")
+    ap.add_argument("--skip-zero-weight", action="store_true",
+                    help="set TLQ_FLAG_SKIP_ZERO_WEIGHT_TOKENS (tensor FLOP/s then count the live tokens only)")
     ap.add_argument("--linears", default=None, help="comma-separated subset of q,k,v,o,gate,up,down (profiling)")
     ap.add_argument("--profile", action="store_true", help="kernel leg only: skip the end-to-end and CPU legs")
     args = ap.parse_args()
