@@ -73,6 +73,12 @@ extern "C" {
                                                w_imp; per_token_err must be NULL.  Losses equal the unflagged call's
                                                up to the order of the fp32 partial sums. */
 
+#define TLQ_FLAG_GEMM_CTA_PAIRS 2u          /* tlq_scale_search_layer, group mode: run the fused GEMM on pairs of CTAs
+                                               (one 256 x 256 MMA per two SMs, the weight tile split between them)
+                                               instead of one CTA per tile.  Same results layout and tolerances.
+                                               Off by default: equal speed in isolation, slower under the power cap
+                                               of a long run on the parts measured. */
+
 #define TLQ_MAX_GRID 64
 
 typedef struct {

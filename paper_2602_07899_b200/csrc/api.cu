@@ -15,7 +15,8 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 int check_cfg(const tlq_config* cfg, int64_t C1, bool need_quantizer = true) {
   if (cfg == nullptr || cfg->struct_size != sizeof(tlq_config)) return TLQ_ERR_INVALID_ARG;
-  if ((cfg->flags & ~(uint32_t)TLQ_FLAG_SKIP_ZERO_WEIGHT_TOKENS) != 0) return TLQ_ERR_INVALID_ARG;
+  if ((cfg->flags & ~(uint32_t)(TLQ_FLAG_SKIP_ZERO_WEIGHT_TOKENS | TLQ_FLAG_GEMM_CTA_PAIRS)) != 0)
+    return TLQ_ERR_INVALID_ARG;
   if (cfg->n_grid < 1 || cfg->n_grid > TLQ_MAX_GRID) return TLQ_ERR_SHAPE;
   if (cfg->stat_mode < TLQ_STAT_MEAN_ABS || cfg->stat_mode > TLQ_STAT_MASKED_MAX) return TLQ_ERR_INVALID_ARG;
   if (C1 < 8 || (C1 % 8) != 0) return TLQ_ERR_SHAPE;
@@ -309,7 +310,12 @@ int tlq_scale_search_layer(const void* X, int64_t N, int64_t C1, const void* W, 
                                      nullptr, st)) != TLQ_OK)
       return rc;
     if ((rc = timing_mark(2, st)) != TLQ_OK) return rc;
-    if ((rc = launch_search_gemm_bf16(Xg, L.dW, wg, L.plan, L.partials, ptab, L.hdr, n_live, st)) != TLQ_OK) return rc;
+    if (cfg->flags & TLQ_FLAG_GEMM_CTA_PAIRS) {
+      if ((rc = launch_search_gemm_bf16_pair(Xg, L.dW, wg, L.plan, L.partials, ptab, L.hdr, n_live, st)) != TLQ_OK)
+        return rc;
+    } else if ((rc = launch_search_gemm_bf16(Xg, L.dW, wg, L.plan, L.partials, ptab, L.hdr, n_live, st)) != TLQ_OK) {
+      return rc;
+    }
   } else {
     if ((rc = launch_fakequant_rows_i8(Wb, L.s, K, C2, C1, cfg->w_bits, L.Wq, L.u, st)) != TLQ_OK) return rc;
     if ((rc = launch_actquant_i8(Xg, nullptr, L.rs, K, N, C1, cfg->a_bits, L.Xq, L.t, n_live, st)) != TLQ_OK) return rc;

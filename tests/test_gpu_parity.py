@@ -465,3 +465,29 @@ def test_skipping_needs_weights_and_has_no_per_token_table(tlq):
     with pytest.raises(tlq.TlqError) as e:
         tlq.tlq_scale_search_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), torch.zeros(64).cuda(), cfg)
     assert e.value.status == tlq.ERR_NONFINITE
+
+
+# ----------------------------------------------------------------------------------- the CTA-pair GEMM
+
+
+@pytest.mark.parametrize("n,c1,c2,group,n_grid", [(256, 512, 512, 128, 20), (300, 288, 320, 32, 5), (130, 128, 100, 64, 3),
+                                                  (1, 64, 8, 32, 2), (515, 1088, 777, 64, 6), (1000, 512, 256, 128, 4)])
+def test_search_on_cta_pairs(tlq, n, c1, c2, group, n_grid):
+    """The same search with the fused GEMM on CTA pairs (256-token tiles across two SMs): oracle parity, and the
+    odd-tile and ragged cases where the second CTA of a pair has no tokens."""
+    xb, wb, imp = wl.small_case(101, n, c1, c2)
+    ref = orc.scale_search(xb, wb, imp, "w4a16", group, n_grid)
+    cfg = tlq.config(group_size=group, n_grid=n_grid, flags=tlq.FLAG_GEMM_CTA_PAIRS)
+    out = tlq.tlq_scale_search_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), torch.from_numpy(imp).cuda(), cfg, per_token=True)
+    got = dict(best=int(out.best_idx.item()), losses=out.losses.cpu().numpy(), per_token=out.per_token.cpu().numpy(),
+               s_best=bits_of(out.s_best))
+    check_against_oracle(got, ref, n_grid)
+    # with token skipping on top (half of the tokens dead)
+    imp2 = imp.copy()
+    imp2[::2] = 0.0
+    if imp2.sum() == 0.0:
+        return
+    ref2 = orc.scale_search(xb, wb, imp2, "w4a16", group, n_grid)
+    cfg2 = tlq.config(group_size=group, n_grid=n_grid, flags=tlq.FLAG_GEMM_CTA_PAIRS | tlq.FLAG_SKIP_ZERO_WEIGHT_TOKENS)
+    out2 = tlq.tlq_scale_search_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), torch.from_numpy(imp2).cuda(), cfg2)
+    np.testing.assert_allclose(out2.losses.cpu().numpy(), ref2["losses"], rtol=LOSS_RTOL)
