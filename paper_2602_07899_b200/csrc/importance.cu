@@ -29,7 +29,23 @@ token_importance_kernel(const void* __restrict__ G, int64_t B, int64_t N, int64_
       }
     } else {
       const uint16_t* g = reinterpret_cast<const uint16_t*>(G) + (b * N + n) * C;
-      for (int64_t c = (int64_t)lane * 8; c < C; c += 32 * 8) {
+      int64_t c = (int64_t)lane * 8;
+      // four 128-bit loads in flight per lane before any is consumed
+      for (; c + 3 * 256 < C; c += 4 * 256) {
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = ld_nc_16(g + c + u * 256);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          float f[8];
+          unpack8(v[u], f);
+          float part = 0.0f;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) part += kL2 ? f[j] * f[j] : fabsf(f[j]);
+          row += (double)part;
+        }
+      }
+      for (; c < C; c += 256) {
         float f[8];
         unpack8(ld_nc_16(g + c), f);
         float part = 0.0f;
