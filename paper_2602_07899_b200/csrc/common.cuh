@@ -104,7 +104,8 @@ struct WorkspaceHeader {
   int32_t status;     // TLQ_OK / TLQ_ERR_TIMEOUT / TLQ_ERR_NONFINITE
   int32_t where;      // diagnostic: which wait gave up
   int32_t best_idx;   // device copy of the argmin
-  int32_t pad[61];
+  int32_t reduce_done; // CTAs of the loss reduction that have finished (the header is zeroed by every call)
+  int32_t pad[60];
 };
 static_assert(sizeof(WorkspaceHeader) == 256, "header is 256 bytes");
 

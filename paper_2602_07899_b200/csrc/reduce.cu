@@ -1,6 +1,6 @@
 // Final reduction of the search: loss[k] = sum_n w_n e_{k,n} / (C2 * sum_n w_n) (the expectation in
 // the objective of paper Sec. 3.2.1 with per-token importance weights), argmin with the lowest index
-// on ties, and the copy of the winning scale row.  Latency-bound: one CTA, fp64, fixed summation
+// on ties, and the copy of the winning scale row.  Latency-bound: one CTA per candidate, fp64, fixed summation
 // order (per-thread strided serial sums, then a binary tree in shared memory), so two runs give
 // bit-identical losses.
 #include "common.cuh"
@@ -21,14 +21,16 @@ __device__ __forceinline__ double block_sum_fixed(double v, double* scratch) {
   return scratch[0];
 }
 
+// One CTA per candidate; the CTA that finishes last takes the argmin and copies the winning scale row.
 __global__ void __launch_bounds__(kRedThreads)
 loss_reduce_kernel(const float* __restrict__ partials, int64_t per_k, int K, const float* __restrict__ w_imp,
                    int64_t N, int64_t C2, const uint16_t* __restrict__ s_table, int64_t C1, WorkspaceHeader* hdr,
                    double* __restrict__ losses, int32_t* __restrict__ best_idx, uint16_t* __restrict__ s_best) {
   __shared__ double scratch[kRedThreads];
-  __shared__ double loss_sh[TLQ_MAX_GRID];
   __shared__ int best_sh;
+  __shared__ int last_sh;
   const int t = threadIdx.x;
+  const int k = blockIdx.x;
 
   double wsum;
   if (w_imp != nullptr) {
@@ -40,24 +42,28 @@ loss_reduce_kernel(const float* __restrict__ partials, int64_t per_k, int K, con
   }
   const double denom = (double)C2 * wsum;
 
-  for (int k = 0; k < K; ++k) {
-    const float* p = partials + (int64_t)k * per_k;
-    double a = 0.0;
-    for (int64_t i = t; i < per_k; i += kRedThreads) a += (double)p[i];
-    const double total = block_sum_fixed(a, scratch);
-    if (t == 0) {
-      double l = total / denom;
-      if (!isfinite(l)) l = __longlong_as_double(0x7FF0000000000000LL);
-      loss_sh[k] = l;
-      losses[k] = l;
-    }
+  const float* p = partials + (int64_t)k * per_k;
+  double a = 0.0;
+  for (int64_t i = t; i < per_k; i += kRedThreads) a += (double)p[i];
+  const double total = block_sum_fixed(a, scratch);
+  if (t == 0) {
+    double l = total / denom;
+    if (!isfinite(l)) l = __longlong_as_double(0x7FF0000000000000LL);
+    losses[k] = l;
+    __threadfence();
+    last_sh = (atomicAdd(&hdr->reduce_done, 1) == K - 1) ? 1 : 0;
   }
   __syncthreads();
+  if (last_sh == 0) return;
+
   if (t == 0) {
+    __threadfence();
     int best = -1;
     double bv = __longlong_as_double(0x7FF0000000000000LL);
-    for (int k = 0; k < K; ++k)
-      if (loss_sh[k] < bv) { bv = loss_sh[k]; best = k; }
+    for (int j = 0; j < K; ++j) {
+      const double lj = __ldcg(losses + j);      // written by other CTAs: read past L1
+      if (lj < bv) { bv = lj; best = j; }
+    }
     if (best < 0) {
       if (hdr->status == TLQ_OK) hdr->status = TLQ_ERR_NONFINITE;
       best = 0;
@@ -86,7 +92,7 @@ __global__ void per_token_reduce_kernel(const float* __restrict__ ptab, int K, i
 int launch_loss_reduce(const float* partials, int64_t per_k, int K, const float* w_imp, int64_t N, int64_t C2,
                        const uint16_t* s_table, int64_t C1, WorkspaceHeader* hdr, double* losses, int32_t* best_idx,
                        uint16_t* s_best, cudaStream_t st) {
-  loss_reduce_kernel<<<1, kRedThreads, 0, st>>>(partials, per_k, K, w_imp, N, C2, s_table, C1, hdr, losses, best_idx,
+  loss_reduce_kernel<<<(unsigned)K, kRedThreads, 0, st>>>(partials, per_k, K, w_imp, N, C2, s_table, C1, hdr, losses, best_idx,
                                                s_best);
   return after_launch();
 }

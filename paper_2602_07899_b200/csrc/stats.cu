@@ -15,7 +15,7 @@ constexpr int kStatTx = 32;   // threads across channels (x8 channels each = 256
 constexpr int kStatTy = 8;    // threads across rows
 
 int64_t stats_row_chunks(int64_t N) {
-  int64_t chunks = ceil_div(N, 64);
+  int64_t chunks = ceil_div(N, 256);      // 32 rows per thread: enough loads in flight, few enough CTAs to launch fast
   if (chunks > 256) chunks = 256;
   if (chunks < 1) chunks = 1;
   return chunks;
@@ -37,7 +37,25 @@ channel_stats_kernel(const uint16_t* __restrict__ X, int64_t N, int64_t C1, cons
   for (int j = 0; j < 8; ++j) acc[j] = 0.0;
 
   if (c0 < C1) {
-    for (int64_t r = r_begin + ty; r < r_end; r += kStatTy) {
+    int64_t r = r_begin + ty;
+    // four rows in flight per thread before any is consumed (a deselected row is loaded and then ignored)
+    for (; r + 3 * kStatTy < r_end; r += 4 * kStatTy) {
+      uint4 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) v[u] = ld_nc_16(X + (r + u * kStatTy) * C1 + c0);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (kMode == TLQ_STAT_MASKED_MAX && mask[r + u * kStatTy] == 0) continue;
+        float f[8];
+        unpack8(v[u], f);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          double a = (double)fabsf(f[j]);
+          if (kMode == TLQ_STAT_MEAN_ABS) acc[j] += a; else acc[j] = fmax(acc[j], a);
+        }
+      }
+    }
+    for (; r < r_end; r += kStatTy) {
       if (kMode == TLQ_STAT_MASKED_MAX && mask[r] == 0) continue;
       float f[8];
       unpack8(ld_nc_16(X + r * C1 + c0), f);
@@ -72,25 +90,26 @@ __device__ __forceinline__ uint16_t double_to_bf16_bits(double x) {
   return (uint16_t)(__float_as_uint((float)r) >> 16);   // r is exactly representable in binary32
 }
 
+// One thread per (channel, candidate): every thread folds the channel's partials in the same fixed order
+// (they sit in L2), then raises the statistic to its own grid power.
 __global__ void scale_table_kernel(const double* __restrict__ partials, int64_t chunks, int64_t N, int64_t C1,
                                    int stat_mode, int K, double* __restrict__ x_stat, uint16_t* __restrict__ s,
                                    float* __restrict__ rs) {
   const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= C1) return;
+  const int k = blockIdx.y * blockDim.y + threadIdx.y;
+  if (c >= C1 || k >= K) return;
   double v = partials[c];
   for (int64_t j = 1; j < chunks; ++j) {
     const double p = partials[j * C1 + c];
     if (stat_mode == TLQ_STAT_MEAN_ABS) v += p; else v = fmax(v, p);
   }
   if (stat_mode == TLQ_STAT_MEAN_ABS) v = v / (double)N;
-  if (x_stat) x_stat[c] = v;
+  if (x_stat != nullptr && k == 0) x_stat[c] = v;
   const double m = fmax(v, kStatFloor);
-  for (int k = 0; k < K; ++k) {
-    const double r = (double)k / (double)K;
-    const uint16_t b = (k == 0) ? (uint16_t)0x3F80 : double_to_bf16_bits(pow(m, r));
-    s[(int64_t)k * C1 + c] = b;
-    if (rs) rs[(int64_t)k * C1 + c] = __fdiv_rn(1.0f, bf16_bits_to_float(b));
-  }
+  const double r = (double)k / (double)K;
+  const uint16_t b = (k == 0) ? (uint16_t)0x3F80 : double_to_bf16_bits(pow(m, r));
+  s[(int64_t)k * C1 + c] = b;
+  if (rs) rs[(int64_t)k * C1 + c] = __fdiv_rn(1.0f, bf16_bits_to_float(b));
 }
 
 int launch_channel_stats(const uint16_t* X, int64_t N, int64_t C1, const uint8_t* mask, int stat_mode,
@@ -114,9 +133,8 @@ int launch_channel_stats(const uint16_t* X, int64_t N, int64_t C1, const uint8_t
 
 int launch_scale_table(const double* partials, int64_t chunks, int64_t N, int64_t C1, int stat_mode, int K,
                        double* x_stat, uint16_t* s, float* rs, cudaStream_t st) {
-  const int threads = 128;
-  scale_table_kernel<<<(unsigned)ceil_div(C1, threads), threads, 0, st>>>(partials, chunks, N, C1, stat_mode, K,
-                                                                         x_stat, s, rs);
+  const dim3 block(32, 8), grid((unsigned)ceil_div(C1, 32), (unsigned)ceil_div(K, 8));
+  scale_table_kernel<<<grid, block, 0, st>>>(partials, chunks, N, C1, stat_mode, K, x_stat, s, rs);
   return after_launch();
 }
 
