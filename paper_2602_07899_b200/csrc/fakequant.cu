@@ -99,9 +99,14 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // lanes: min/max go through xor-shuffles.  grid.z splits the candidates when the matrix alone
 // would not fill the machine.
 // ------------------------------------------------------------------------------------------------
-constexpr int kGqRows = 32;
+constexpr int kGqRows = 32;      // tile height of the general one-scale kernel (static shared memory)
+constexpr int kHotRows = 64;     // tile height of the delta-weight kernel: 64 KB of dynamic shared memory, so the
+                                 // per-candidate scale tables are fetched once per 8 rows of a warp, not per 4
 constexpr int kGqCols = 512;
 constexpr int kGqThreads = 256;
+constexpr size_t kHotSmem = (size_t)kHotRows * kGqCols * 2;
+constexpr int kRowRows = 32;     // row quantizers: 32 KB tiles leave the L1 to the per-candidate reciprocal tables (64-row tiles measured slower)
+constexpr size_t kRowSmem = (size_t)kRowRows * kGqCols * 2;
 
 // ------------------------------------------------------------------------------------------------
 // The search's own fake-quant pass: delta weights of ALL candidates, nothing else.  Same tile and
@@ -147,11 +152,12 @@ __global__ void __launch_bounds__(kGqThreads, 2)
 fakequant_delta_kernel(const uint16_t* __restrict__ W, const uint16_t* __restrict__ s_tab,
                        const float* __restrict__ rs_tab, int K, int k_per_cta, int64_t C2, int64_t C1, int group,
                        int qmax, float tie_eps, uint16_t* __restrict__ dW) {
-  __shared__ uint4 tile[kGqRows][kGqCols / 8];
+  extern __shared__ uint4 tile_dyn[];
+  uint4 (*tile)[kGqCols / 8] = reinterpret_cast<uint4 (*)[kGqCols / 8]>(tile_dyn);
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const int64_t c0 = (int64_t)blockIdx.x * kGqCols + lane * 16;
-  const int64_t row0 = (int64_t)blockIdx.y * kGqRows;
+  const int64_t row0 = (int64_t)blockIdx.y * kHotRows;
   const bool col_ok = c0 < C1;
   const int lanes_per_group = group >> 4;
   const float qmax_f = (float)qmax;
@@ -160,7 +166,7 @@ fakequant_delta_kernel(const uint16_t* __restrict__ W, const uint16_t* __restric
   const int k_end = min(K, k_begin + k_per_cta);
 
 #pragma unroll
-  for (int p = 0; p < kGqRows / 8; ++p) {
+  for (int p = 0; p < kHotRows / 8; ++p) {
     const int r = p * 8 + warp;
     uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0;
     if (col_ok && row0 + r < C2) {
@@ -193,7 +199,7 @@ fakequant_delta_kernel(const uint16_t* __restrict__ W, const uint16_t* __restric
       }
     }
 #pragma unroll 1
-    for (int p = 0; p < kGqRows / 8; ++p) {
+    for (int p = 0; p < kHotRows / 8; ++p) {
       const int r = p * 8 + warp;
       const int64_t row = row0 + r;
       if (row >= C2) break;                       // rows of a warp ascend with p; shuffles below stay warp-uniform
@@ -393,18 +399,26 @@ fakequant_group_kernel(const uint16_t* __restrict__ W, const uint16_t* __restric
 int launch_fakequant_group(const uint16_t* W, const uint16_t* s, const float* rs, int K, int64_t C2, int64_t C1,
                            int group, int w_bits, uint16_t* dW, uint8_t* codes, float* steps, int32_t* zeros,
                            cudaStream_t st) {
-  const int64_t ctas = ceil_div(C1, kGqCols) * ceil_div(C2, kGqRows);
+  const bool hot = dW != nullptr && s != nullptr && rs != nullptr && codes == nullptr && steps == nullptr && zeros == nullptr;
+  const int tile_rows = hot ? kHotRows : kGqRows;
+  const int64_t ctas = ceil_div(C1, kGqCols) * ceil_div(C2, tile_rows);
   int64_t kchunks = ceil_div(148 * 6, ctas);        // aim for several CTAs per SM
   if (kchunks > K) kchunks = K;
   if (kchunks < 1) kchunks = 1;
   const int k_per_cta = (int)ceil_div(K, kchunks);
   kchunks = ceil_div(K, k_per_cta);
-  dim3 grid((unsigned)ceil_div(C1, kGqCols), (unsigned)ceil_div(C2, kGqRows), (unsigned)kchunks);
-  if (dW != nullptr && s != nullptr && rs != nullptr && codes == nullptr && steps == nullptr && zeros == nullptr) {
+  dim3 grid((unsigned)ceil_div(C1, kGqCols), (unsigned)ceil_div(C2, tile_rows), (unsigned)kchunks);
+  if (hot) {
+    static bool configured = false;
+    if (!configured) {
+      TLQ_CUDA_TRY(cudaFuncSetAttribute(fakequant_delta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)kHotSmem));
+      configured = true;
+    }
     // |quotient| <= qmax + 1 on the straight-line path; 4e-7 per unit covers the reciprocal (1 ulp), the product
     // and the exact quotient's own rounding (together < 2.4e-7 relative)
     const float tie_eps = 4.0e-7f * (float)(1 << w_bits);
-    fakequant_delta_kernel<<<grid, kGqThreads, 0, st>>>(W, s, rs, K, k_per_cta, C2, C1, group, (1 << w_bits) - 1,
+    fakequant_delta_kernel<<<grid, kGqThreads, kHotSmem, st>>>(W, s, rs, K, k_per_cta, C2, C1, group, (1 << w_bits) - 1,
                                                         tie_eps, dW);
     return after_launch();
   }
@@ -464,7 +478,7 @@ __device__ __forceinline__ void load_mult16(const uint16_t* s_row, const float* 
 __device__ __forceinline__ void stage_tile(uint4 (*tile)[kGqCols / 8], const uint16_t* __restrict__ src, int64_t row0,
                                            int64_t R, int64_t C1, int64_t c0, bool col_ok, int warp, int lane) {
 #pragma unroll
-  for (int p = 0; p < kGqRows / 8; ++p) {
+  for (int p = 0; p < kRowRows / 8; ++p) {
     const int r = p * 8 + warp;
     uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0;
     if (col_ok && row0 + r < R) {
@@ -488,10 +502,11 @@ __global__ void __launch_bounds__(kGqThreads, 3)
 row_amax_kernel(const uint16_t* __restrict__ src, const uint16_t* __restrict__ s_tab, const float* __restrict__ rs_tab,
                 int K, int k_per_cta, int64_t R_all, const int32_t* __restrict__ n_rows_dev, int64_t C1,
                 int* __restrict__ amax_bits /*[K,R_all], zeroed*/) {
-  __shared__ uint4 tile[kGqRows][kGqCols / 8];
+  extern __shared__ uint4 tile_dyn[];
+  uint4 (*tile)[kGqCols / 8] = reinterpret_cast<uint4 (*)[kGqCols / 8]>(tile_dyn);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t c0 = (int64_t)blockIdx.x * kGqCols + lane * 16;
-  const int64_t row0 = (int64_t)blockIdx.y * kGqRows;
+  const int64_t row0 = (int64_t)blockIdx.y * kRowRows;
   const int64_t R = (n_rows_dev != nullptr) ? (int64_t)*n_rows_dev : R_all;    // rows beyond are not live
   if (row0 >= R) return;                                                        // the whole CTA leaves together
   const bool col_ok = c0 < C1;
@@ -502,21 +517,32 @@ row_amax_kernel(const uint16_t* __restrict__ src, const uint16_t* __restrict__ s
     float2 m[8];
     load_mult16<kKind>(s_tab ? s_tab + (int64_t)k * C1 : nullptr, rs_tab ? rs_tab + (int64_t)k * C1 : nullptr, c0,
                        col_ok, m);
+    // four of the warp's rows at a time: four independent shuffle chains instead of one after the other
 #pragma unroll 1
-    for (int p = 0; p < kGqRows / 8; ++p) {
-      const int r = p * 8 + warp;
-      if (row0 + r >= R) break;
-      float2 w[8];
-      unpack16(tile[r][lane * 2], tile[r][lane * 2 + 1], w);
-      float a = 0.0f;
+    for (int h = 0; h < kRowRows / 32; ++h) {
+      float a[4];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const float2 v = mul2(w[j], m[j]);
-        a = max3(a, fabsf(v.x), fabsf(v.y));
+      for (int p = 0; p < 4; ++p) {
+        const int r = (h * 4 + p) * 8 + warp;          // rows past the end were staged as zeros
+        float2 w[8];
+        unpack16(tile[r][lane * 2], tile[r][lane * 2 + 1], w);
+        a[p] = 0.0f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const float2 v = mul2(w[j], m[j]);
+          a[p] = max3(a[p], fabsf(v.x), fabsf(v.y));
+        }
       }
 #pragma unroll
-      for (int off = 16; off > 0; off >>= 1) a = fmaxf(a, __shfl_xor_sync(0xFFFFFFFFu, a, off));
-      if (lane == 0) atomicMax(amax_bits + (int64_t)k * R_all + row0 + r, __float_as_int(a));
+      for (int off = 16; off > 0; off >>= 1) {
+#pragma unroll
+        for (int p = 0; p < 4; ++p) a[p] = fmaxf(a[p], __shfl_xor_sync(0xFFFFFFFFu, a[p], off));
+      }
+      float mine = a[0];
+#pragma unroll
+      for (int p = 1; p < 4; ++p) mine = (lane == p) ? a[p] : mine;
+      const int64_t my_row = row0 + (h * 4 + lane) * 8 + warp;
+      if (lane < 4 && my_row < R) atomicMax(amax_bits + (int64_t)k * R_all + my_row, __float_as_int(mine));
     }
   }
 }
@@ -550,10 +576,11 @@ row_codes_kernel(const uint16_t* __restrict__ src, const uint16_t* __restrict__ 
                  const float* __restrict__ step /*[K,R_all]*/, int K, int k_per_cta, int64_t R_all,
                  const int32_t* __restrict__ n_rows_dev, int64_t C1, float qpos, float tie_eps,
                  int8_t* __restrict__ q /*[K,R_all,C1]*/) {
-  __shared__ uint4 tile[kGqRows][kGqCols / 8];
+  extern __shared__ uint4 tile_dyn[];
+  uint4 (*tile)[kGqCols / 8] = reinterpret_cast<uint4 (*)[kGqCols / 8]>(tile_dyn);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t c0 = (int64_t)blockIdx.x * kGqCols + lane * 16;
-  const int64_t row0 = (int64_t)blockIdx.y * kGqRows;
+  const int64_t row0 = (int64_t)blockIdx.y * kRowRows;
   const int64_t R = (n_rows_dev != nullptr) ? (int64_t)*n_rows_dev : R_all;
   if (row0 >= R) return;
   const bool col_ok = c0 < C1;
@@ -568,7 +595,7 @@ row_codes_kernel(const uint16_t* __restrict__ src, const uint16_t* __restrict__ 
     load_mult16<kKind>(s_tab ? s_tab + (int64_t)k * C1 : nullptr, rs_tab ? rs_tab + (int64_t)k * C1 : nullptr, c0,
                        true, m);
 #pragma unroll 1
-    for (int p = 0; p < kGqRows / 8; ++p) {
+    for (int p = 0; p < kRowRows / 8; ++p) {
       const int r = p * 8 + warp;
       const int64_t row = row0 + r;
       if (row >= R) break;
@@ -609,24 +636,30 @@ row_codes_kernel(const uint16_t* __restrict__ src, const uint16_t* __restrict__ 
 template <int kKind>
 static int launch_rows(const uint16_t* src, const uint16_t* s, const float* rs, int K, int64_t R, int64_t C1, int bits,
                        int8_t* q, float* step, const int32_t* n_rows_dev, cudaStream_t st) {
-  const int64_t ctas = ceil_div(C1, kGqCols) * ceil_div(R, kGqRows);
+  static bool configured = false;      // one flag per instantiation of this template
+  if (!configured) {
+    TLQ_CUDA_TRY(cudaFuncSetAttribute(row_amax_kernel<kKind>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kRowSmem));
+    TLQ_CUDA_TRY(cudaFuncSetAttribute(row_codes_kernel<kKind>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kRowSmem));
+    configured = true;
+  }
+  const int64_t ctas = ceil_div(C1, kGqCols) * ceil_div(R, kRowRows);
   int64_t kchunks = ceil_div(148 * 6, ctas);
   if (kchunks > K) kchunks = K;
   if (kchunks < 1) kchunks = 1;
   const int k_per_cta = (int)ceil_div(K, kchunks);
   kchunks = ceil_div(K, k_per_cta);
-  const dim3 grid((unsigned)ceil_div(C1, kGqCols), (unsigned)ceil_div(R, kGqRows), (unsigned)kchunks);
+  const dim3 grid((unsigned)ceil_div(C1, kGqCols), (unsigned)ceil_div(R, kRowRows), (unsigned)kchunks);
   const float qpos = (float)((1 << (bits - 1)) - 1);
   const float tie_eps = 4.0e-7f * (qpos + 1.0f);
   const int64_t n = (int64_t)K * R;
   TLQ_CUDA_TRY(cudaMemsetAsync(step, 0, (size_t)n * sizeof(float), st));
-  row_amax_kernel<kKind><<<grid, kGqThreads, 0, st>>>(src, s, rs, K, k_per_cta, R, n_rows_dev, C1,
+  row_amax_kernel<kKind><<<grid, kGqThreads, kRowSmem, st>>>(src, s, rs, K, k_per_cta, R, n_rows_dev, C1,
                                                       reinterpret_cast<int*>(step));
   int rc = after_launch();
   if (rc != TLQ_OK) return rc;
   amax_to_step_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(step, n, qpos);
   if ((rc = after_launch()) != TLQ_OK) return rc;
-  row_codes_kernel<kKind><<<grid, kGqThreads, 0, st>>>(src, s, rs, step, K, k_per_cta, R, n_rows_dev, C1, qpos, tie_eps, q);
+  row_codes_kernel<kKind><<<grid, kGqThreads, kRowSmem, st>>>(src, s, rs, step, K, k_per_cta, R, n_rows_dev, C1, qpos, tie_eps, q);
   return after_launch();
 }
 
