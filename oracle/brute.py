@@ -51,13 +51,16 @@ def nearest_level(p: float, step: float, zero: int, qmax: int) -> list[int]:
     return arg
 
 
-def search(x_bits, w_bits, w_imp, group: int, n_grid: int, bits: int = 4, mode: str = "w4a16"):
-    """Exhaustive scale search on nested lists; returns (best index, losses list, per-token table)."""
+def search(x_bits, w_bits, w_imp, group: int, n_grid: int, bits: int = 4, mode: str = "w4a16", x_fp_bits=None):
+    """Exhaustive scale search on nested lists; returns (best index, losses list, per-token table).
+    `x_fp_bits`: the full-precision stream of the two-stream objective (the reference output is computed
+    from it, everything on the quantized side from x_bits)."""
     n, c1, c2 = len(x_bits), len(x_bits[0]), len(w_bits)
     x = [[bf16_value(v) for v in row] for row in x_bits]
+    x_ref = x if x_fp_bits is None else [[bf16_value(v) for v in row] for row in x_fp_bits]
     w = [[bf16_value(v) for v in row] for row in w_bits]
     stat = [max(sum(abs(x[i][c]) for i in range(n)) / n, 2.0 ** -20) for c in range(c1)]
-    y_fp = [[sum(w[o][c] * x[i][c] for c in range(c1)) for o in range(c2)] for i in range(n)]
+    y_fp = [[sum(w[o][c] * x_ref[i][c] for c in range(c1)) for o in range(c2)] for i in range(n)]
     qmax = (1 << bits) - 1
     losses, table = [], []
     for k in range(n_grid):

@@ -272,17 +272,22 @@ def candidate_error(x_bits, w_bits, s_k, mode: str, group: int, y_fp: np.ndarray
 
 def scale_search(x_bits: np.ndarray, w_bits: np.ndarray, w_imp: np.ndarray | None, mode: str = "w4a16",
                  group: int = 128, n_grid: int = 20, stat_mode: int = STAT_MEAN_ABS,
-                 mask: np.ndarray | None = None, w_bits_n: int = 4):
+                 mask: np.ndarray | None = None, w_bits_n: int = 4, x_fp_bits: np.ndarray | None = None):
     """The layer-wise search of Sec. 3.2.1 over the grid r_k = k/K, in the paper's order:
     x_stat -> scale(r) -> quantize the scaled weights (and smoothed activations) -> apply the
     quantized layer to the calibration tokens -> squared output error per token -> importance-
     weighted mean -> argmin.
 
+    `x_fp_bits` selects the paper's first propagation strategy (Sec. 3.2.1, PassAct1): two activation
+    streams, the full-precision layer sees x_fp (output of the full-precision layers before it) while the
+    quantized layer, and the statistic behind its scale, see `x_bits` (output of the already quantized
+    layers): loss = || f_fp(x_fp) - f_q(x_q; scale) ||^2.  Without it both see `x_bits`.
+
     Returns dict(best, losses float64 [K], per_token float64 [K,N], scales float32 [K,C1], x_stat).
     """
     x_stat = channel_stat(x_bits, stat_mode, mask)
     scales = scale_table(x_stat, n_grid)
-    y_fp = layer_fp(x_bits, w_bits)
+    y_fp = layer_fp(x_bits if x_fp_bits is None else x_fp_bits, w_bits)
     c_out = w_bits.shape[0]
     per_token = np.empty((n_grid, x_bits.shape[0]), dtype=F64)
     losses = np.empty(n_grid, dtype=F64)

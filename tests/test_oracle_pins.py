@@ -415,3 +415,27 @@ def test_shared_scale_of_sibling_linears_is_the_search_on_stacked_rows():
         assert np.allclose(c["per_token"], a["per_token"] + b["per_token"], rtol=1e-12)
         assert np.allclose(c["losses"], (24 * a["losses"] + 8 * b["losses"]) / 32, rtol=1e-12)
         assert np.array_equal(c["scales"], a["scales"])
+
+
+@pytest.mark.parametrize("mode", ["w4a16", "w4a8"])
+def test_two_stream_objective(mode):
+    """First propagation strategy of Sec. 3.2.1: || f_fp(x_fp) - f_q(x_q) ||^2.  With equal streams it is the
+    plain search; in general the error splits into a candidate-independent part (x_fp - x_q) W^T plus the
+    single-stream error term, checked through that second route and against the scalar brute force."""
+    xq, w, imp = wl.small_case(111, 6, 8, 3)
+    xf, _, _ = wl.small_case(112, 6, 8, 3)
+    same = orc.scale_search(xq, w, imp, mode=mode, group=4, n_grid=3, x_fp_bits=xq)
+    plain = orc.scale_search(xq, w, imp, mode=mode, group=4, n_grid=3)
+    assert np.array_equal(same["per_token"], plain["per_token"]) and same["best"] == plain["best"]
+    two = orc.scale_search(xq, w, imp, mode=mode, group=4, n_grid=3, x_fp_bits=xf)
+    assert np.array_equal(two["scales"], plain["scales"])          # the scale follows the quantized stream
+    best, losses, table = brute.search(xq.tolist(), w.tolist(), [float(v) for v in imp], 4, 3, 4, mode, xf.tolist())
+    assert best == two["best"]
+    assert np.allclose(losses, two["losses"], rtol=1e-11)
+    assert np.allclose(np.array(table), two["per_token"], rtol=1e-11, atol=1e-18)
+    if mode == "w4a16":
+        d = (orc.bf16_to_f64(xf) - orc.bf16_to_f64(xq)) @ orc.bf16_to_f64(w).T
+        for k in range(3):
+            _, _, _, w_hat = orc.quantize_weights_group_asym(w, two["scales"][k], 4)
+            e = d + orc.bf16_to_f64(xq) @ (orc.bf16_to_f64(w) - w_hat.astype(np.float64)).T
+            assert np.allclose(two["per_token"][k], (e ** 2).sum(axis=1), rtol=1e-9)
