@@ -182,6 +182,19 @@ int tlq_scale_search_layer(const void* X, int64_t N, int64_t C1, const void* W, 
                            float* per_token_err, void* stream);
 
 /*
+ * The same search under the paper's first propagation strategy (Sec. 3.2.1, PassAct1): two activation streams.
+ * X_fp [N,C1] bf16 is the layer's input as the full-precision layers before it produce it, X_q [N,C1] bf16 its input
+ * as the already quantized layers produce it; e_{k,n} = || f_fp(x_fp,n) - f_q(x_q,n; scale_k) ||_2^2.  The scale
+ * statistic, the smoothing and the activation quantizer all act on X_q.  Everything else as in
+ * tlq_scale_search_layer (same workspace size); the flags TLQ_FLAG_SKIP_ZERO_WEIGHT_TOKENS and
+ * TLQ_FLAG_GEMM_CTA_PAIRS are not accepted here.
+ */
+int tlq_scale_search_layer_two_stream(const void* X_q, const void* X_fp, int64_t N, int64_t C1, const void* W,
+                                      int64_t C2, const float* w_imp, const uint8_t* mask, const tlq_config* cfg,
+                                      void* workspace, size_t workspace_bytes, int32_t* best_idx, double* losses,
+                                      void* s_best, float* per_token_err, void* stream);
+
+/*
  * Apply the quantized layer with a chosen scale: Y_q = f_q(X; s) (+ bias), the activation the next
  * layer calibrates on under the paper's adopted propagation strategy (Sec. 3.2.1, PassAct2).
  *   s [C1] bf16 or NULL; bias [C2] bf16 or NULL; Yq [N,C2] bf16 (C2 a multiple of 8);

@@ -76,8 +76,9 @@ struct SearchLayout {
   float* wc;             // [n_pad] packed weights
   uint16_t* Xc;          // [n_pad, C1] packed activations
   size_t bytes;
-  GemmPlan plan;
-  int64_t ptab_slices;   // per-candidate slices of the per-token table (column tiles, x2 for W8A8)
+  GemmPlan plan;         // the mode's own GEMM
+  GemmPlan plan_resident; // the tile-resident kernel's (all candidates per tile): symmetric modes and the two-stream search
+  int64_t ptab_slices;   // per-candidate slices of the per-token table as the buffers are sized (2 per column tile)
 };
 
 SearchLayout carve_search(void* ws, int64_t N, int64_t C1, int64_t C2, const tlq_config* cfg) {
@@ -85,14 +86,15 @@ SearchLayout carve_search(void* ws, int64_t N, int64_t C1, int64_t C2, const tlq
   const int K = cfg->n_grid;
   Carver c(ws);
   const bool i8 = cfg->mode == TLQ_W8A8_SYM;
-  L.plan = i8 ? plan_search_gemm_i8(N, C1, C2, K) : plan_search_gemm(N, C1, C2, K);
-  L.ptab_slices = L.plan.otiles * (i8 ? 2 : 1);
+  L.plan_resident = plan_search_gemm_i8(N, C1, C2, K);
+  L.plan = i8 ? L.plan_resident : plan_search_gemm(N, C1, C2, K);
+  L.ptab_slices = L.plan.otiles * 2;
   L.hdr = c.take<WorkspaceHeader>(1);
   L.stat_partials = c.take<double>((size_t)stats_row_chunks(N) * C1);
   L.x_stat = c.take<double>((size_t)C1);
   L.s = c.take<uint16_t>((size_t)K * C1);
   L.rs = c.take<float>((size_t)K * C1);
-  L.partials = c.take<float>((size_t)K * L.plan.partials_per_k);
+  L.partials = c.take<float>((size_t)K * L.plan_resident.partials_per_k);
   L.ptab = c.take<float>((size_t)K * L.ptab_slices * L.plan.n_pad);
   if (cfg->mode == TLQ_W4A16_ASYM_GROUP) {
     L.dW = c.take<uint16_t>((size_t)K * C2 * C1, 1024);
@@ -265,9 +267,14 @@ size_t tlq_scale_search_workspace_bytes(int64_t N, int64_t C1, int64_t C2, const
   return carve_search(nullptr, N, C1, C2, cfg).bytes;
 }
 
-int tlq_scale_search_layer(const void* X, int64_t N, int64_t C1, const void* W, int64_t C2, const float* w_imp,
-                           const uint8_t* mask, const tlq_config* cfg, void* workspace, size_t workspace_bytes,
-                           int32_t* best_idx, double* losses, void* s_best, float* per_token_err, void* stream) {
+}  // extern "C"
+
+// X is what the quantized layer (and the scale statistic) sees; X_ref, when given, is what the full-precision
+// layer sees (two-stream objective).
+static int search_impl(const void* X, const void* X_ref, int64_t N, int64_t C1, const void* W, int64_t C2,
+                       const float* w_imp, const uint8_t* mask, const tlq_config* cfg, void* workspace,
+                       size_t workspace_bytes, int32_t* best_idx, double* losses, void* s_best, float* per_token_err,
+                       void* stream) {
   if (X == nullptr || W == nullptr || workspace == nullptr || best_idx == nullptr || losses == nullptr)
     return TLQ_ERR_INVALID_ARG;
   if (N < 1 || C2 < 1 || N > 0x7FFFFF00LL || C2 > 0x7FFFFF00LL) return TLQ_ERR_SHAPE;
@@ -277,7 +284,10 @@ int tlq_scale_search_layer(const void* X, int64_t N, int64_t C1, const void* W, 
   // skipping needs weights to look at; per-token errors of skipped tokens would not exist
   const bool compact = (cfg->flags & TLQ_FLAG_SKIP_ZERO_WEIGHT_TOKENS) != 0;
   if (compact && (w_imp == nullptr || per_token_err != nullptr)) return TLQ_ERR_INVALID_ARG;
-  if (!aligned16(X) || !aligned16(W) || !aligned16(workspace)) return TLQ_ERR_ALIGN;
+  const bool two_stream = X_ref != nullptr;
+  if (two_stream && (cfg->flags & (TLQ_FLAG_SKIP_ZERO_WEIGHT_TOKENS | TLQ_FLAG_GEMM_CTA_PAIRS)) != 0)
+    return TLQ_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(W) || !aligned16(workspace) || !aligned16(X_ref)) return TLQ_ERR_ALIGN;
   SearchLayout L = carve_search(workspace, N, C1, C2, cfg);
   if (workspace_bytes < L.bytes) return TLQ_ERR_WORKSPACE;
   rc = have_device();
@@ -302,7 +312,7 @@ int tlq_scale_search_layer(const void* X, int64_t N, int64_t C1, const void* W, 
   if (compact) {
     if ((rc = launch_compact_tokens(Xb, w_imp, N, L.plan.n_pad, C1, L.live_idx, L.wc, L.live, L.Xc, st)) != TLQ_OK)
       return rc;
-    TLQ_CUDA_TRY(cudaMemsetAsync(L.partials, 0, (size_t)K * L.plan.partials_per_k * sizeof(float), st));
+    TLQ_CUDA_TRY(cudaMemsetAsync(L.partials, 0, (size_t)K * L.plan_resident.partials_per_k * sizeof(float), st));
     Xg = L.Xc; wg = L.wc; n_live = L.live;
   }
   if (cfg->mode == TLQ_W4A16_ASYM_GROUP) {
@@ -310,7 +320,11 @@ int tlq_scale_search_layer(const void* X, int64_t N, int64_t C1, const void* W, 
                                      nullptr, st)) != TLQ_OK)
       return rc;
     if ((rc = timing_mark(2, st)) != TLQ_OK) return rc;
-    if (cfg->flags & TLQ_FLAG_GEMM_CTA_PAIRS) {
+    if (two_stream) {
+      if ((rc = launch_search_gemm_dual_bf16(Xb, reinterpret_cast<const uint16_t*>(X_ref), Wb, L.dW, w_imp,
+                                             L.plan_resident, L.partials, ptab, L.hdr, st)) != TLQ_OK)
+        return rc;
+    } else if (cfg->flags & TLQ_FLAG_GEMM_CTA_PAIRS) {
       if ((rc = launch_search_gemm_bf16_pair(Xg, L.dW, wg, L.plan, L.partials, ptab, L.hdr, n_live, st)) != TLQ_OK)
         return rc;
     } else if ((rc = launch_search_gemm_bf16(Xg, L.dW, wg, L.plan, L.partials, ptab, L.hdr, n_live, st)) != TLQ_OK) {
@@ -320,19 +334,43 @@ int tlq_scale_search_layer(const void* X, int64_t N, int64_t C1, const void* W, 
     if ((rc = launch_fakequant_rows_i8(Wb, L.s, K, C2, C1, cfg->w_bits, L.Wq, L.u, st)) != TLQ_OK) return rc;
     if ((rc = launch_actquant_i8(Xg, nullptr, L.rs, K, N, C1, cfg->a_bits, L.Xq, L.t, n_live, st)) != TLQ_OK) return rc;
     if ((rc = timing_mark(2, st)) != TLQ_OK) return rc;
-    if ((rc = launch_search_gemm_i8(Xg, Wb, L.Xq, L.Wq, L.t, L.u, wg, L.plan, L.partials, ptab, L.hdr, n_live, st)) !=
+    // the full-precision tile comes from the reference stream when there is one (compaction excludes that case)
+    const uint16_t* Xfp = two_stream ? reinterpret_cast<const uint16_t*>(X_ref) : Xg;
+    if ((rc = launch_search_gemm_i8(Xfp, Wb, L.Xq, L.Wq, L.t, L.u, wg, L.plan, L.partials, ptab, L.hdr, n_live, st)) !=
         TLQ_OK)
       return rc;
   }
   if ((rc = timing_mark(3, st)) != TLQ_OK) return rc;
-  if ((rc = launch_loss_reduce(L.partials, L.plan.partials_per_k, K, w_imp, N, C2, L.s, C1, L.hdr, losses, best_idx,
+  const bool resident = two_stream || cfg->mode != TLQ_W4A16_ASYM_GROUP;
+  const GemmPlan& used = resident ? L.plan_resident : L.plan;
+  if ((rc = launch_loss_reduce(L.partials, used.partials_per_k, K, w_imp, N, C2, L.s, C1, L.hdr, losses, best_idx,
                                reinterpret_cast<uint16_t*>(s_best), st)) != TLQ_OK)
     return rc;
   if (per_token_err != nullptr)
-    if ((rc = launch_per_token_reduce(L.ptab, K, L.ptab_slices, L.plan.n_pad, N, per_token_err, st)) != TLQ_OK)
+    if ((rc = launch_per_token_reduce(L.ptab, K, used.otiles * (resident ? 2 : 1), used.n_pad, N, per_token_err, st)) != TLQ_OK)
       return rc;
   return timing_mark(4, st);
 }
+
+extern "C" {
+
+int tlq_scale_search_layer(const void* X, int64_t N, int64_t C1, const void* W, int64_t C2, const float* w_imp,
+                           const uint8_t* mask, const tlq_config* cfg, void* workspace, size_t workspace_bytes,
+                           int32_t* best_idx, double* losses, void* s_best, float* per_token_err, void* stream) {
+  return search_impl(X, nullptr, N, C1, W, C2, w_imp, mask, cfg, workspace, workspace_bytes, best_idx, losses, s_best,
+                     per_token_err, stream);
+}
+
+int tlq_scale_search_layer_two_stream(const void* X_q, const void* X_fp, int64_t N, int64_t C1, const void* W,
+                                      int64_t C2, const float* w_imp, const uint8_t* mask, const tlq_config* cfg,
+                                      void* workspace, size_t workspace_bytes, int32_t* best_idx, double* losses,
+                                      void* s_best, float* per_token_err, void* stream) {
+  if (X_fp == nullptr) return TLQ_ERR_INVALID_ARG;
+  return search_impl(X_q, X_fp, N, C1, W, C2, w_imp, mask, cfg, workspace, workspace_bytes, best_idx, losses, s_best,
+                     per_token_err, stream);
+}
+
+}  // extern "C"
 
 namespace {
 struct ApplyLayout {
@@ -360,6 +398,8 @@ ApplyLayout carve_apply(void* ws, int64_t N, int64_t C1, int64_t C2, const tlq_c
   return L;
 }
 }  // namespace
+
+extern "C" {
 
 size_t tlq_apply_layer_workspace_bytes(int64_t N, int64_t C1, int64_t C2, const tlq_config* cfg) {
   if (N < 1 || C2 < 1 || check_cfg(cfg, C1) != TLQ_OK) return 0;

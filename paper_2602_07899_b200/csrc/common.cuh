@@ -183,6 +183,10 @@ GemmPlan plan_search_gemm_i8(int64_t N, int64_t C1, int64_t C2, int K);   // par
 int launch_search_gemm_i8(const uint16_t* X, const uint16_t* W, const int8_t* Xq, const int8_t* Wq, const float* t,
                           const float* u, const float* w_imp, const GemmPlan& plan, float* partials, float* ptab,
                           WorkspaceHeader* hdr, const int32_t* n_live, cudaStream_t st);
+// Two-stream search with 16-bit activations (reference from Xfp, quantized side from Xq); plan = plan_search_gemm_i8
+int launch_search_gemm_dual_bf16(const uint16_t* Xq, const uint16_t* Xfp, const uint16_t* W, const uint16_t* dW,
+                                 const float* w_imp, const GemmPlan& plan, float* partials, float* ptab,
+                                 WorkspaceHeader* hdr, cudaStream_t st);
 // Apply: Yq[N,C2] = t[n] * u[o] * (Xq Wq^T) (+bias), bf16 out
 int launch_apply_gemm_i8(const int8_t* Xq, const int8_t* Wq, const float* t, const float* u, const uint16_t* bias,
                          int64_t N, int64_t C1, int64_t C2, uint16_t* Yq, WorkspaceHeader* hdr, cudaStream_t st);

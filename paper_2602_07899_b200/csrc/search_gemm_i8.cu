@@ -39,6 +39,7 @@ constexpr uint32_t kTmemCols = 512;
 constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 256;
 
 constexpr uint32_t kIdescBf16 = ptx::make_idesc(1, 1, BM, BN, false);   // bf16 x bf16 -> f32
+constexpr uint32_t kIdescBf16NegB = ptx::make_idesc(1, 1, BM, BN, true);
 constexpr uint32_t kIdescI8 = ptx::make_idesc(2, 1, BM, BN, false);     // s8 x s8 -> s32
 
 struct I8Args {
@@ -65,7 +66,14 @@ __device__ __forceinline__ void report_timeout(WorkspaceHeader* hdr, int where) 
   hdr->status = TLQ_ERR_TIMEOUT;
 }
 
-template <bool kApply>
+// kMode 0: W8A8-style search (one bf16 pass for the full-precision tile, then K int8 passes)
+// kMode 1: apply (a single int8 pass, bf16 store)
+// kMode 2: two-stream search with 16-bit activations (first propagation strategy of paper Sec. 3.2.1):
+//          || f_fp(x_fp) - f_q(x_q) ||^2 with f_fp - f_q = (X_fp - X_q) W^T + X_q dW_k^T.  The candidate-free
+//          part is accumulated once per tile by two bf16 passes into one accumulator (X_fp W^T, then X_q W^T
+//          with the negate bit) and kept in registers; every candidate adds its bf16 pass X_q dW_k^T to it.
+//          Tensor maps: tmX = X_fp, tmW = W, tmXq = X_q (bf16, 3-D with a single slice), tmWq = dW (bf16, 3-D).
+template <int kMode>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_w8a8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW,
                  const __grid_constant__ CUtensorMap tmXq, const __grid_constant__ CUtensorMap tmWq,
@@ -82,6 +90,8 @@ gemm_w8a8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr bool kApply = kMode == 1;
+  constexpr bool kDual = kMode == 2;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -130,7 +140,7 @@ gemm_w8a8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         for (int pass = 0; pass < passes && ok; ++pass) {
           const bool fp = !kApply && pass == 0;
           const int k = kApply ? 0 : pass - 1;
-          const int nkb = fp ? args.num_kb16 : args.num_kb8;
+          const int nkb = fp ? (kDual ? 2 * args.num_kb16 : args.num_kb16) : (kDual ? args.num_kb16 : args.num_kb8);
           for (int kb = 0; kb < nkb; ++kb) {
             if (!ptx::mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
               report_timeout(args.hdr, 11);
@@ -139,9 +149,16 @@ gemm_w8a8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             }
             const uint32_t a_dst = smem_base + stage * kStageBytes;
             ptx::mbar_expect_tx(full_bar(stage), kStageBytes);
-            if (fp) {
+            if (fp && kDual && kb >= args.num_kb16) {        // second half of the reference pass: X_q against W
+              const int kq = kb - args.num_kb16;
+              ptx::tma_load_3d(a_dst, &tmXq, full_bar(stage), kq * BK16, mt * BM, 0);
+              ptx::tma_load_2d(a_dst + kABytes, &tmW, full_bar(stage), kq * BK16, ot * BN);
+            } else if (fp) {
               ptx::tma_load_2d(a_dst, &tmX, full_bar(stage), kb * BK16, mt * BM);
               ptx::tma_load_2d(a_dst + kABytes, &tmW, full_bar(stage), kb * BK16, ot * BN);
+            } else if (kDual) {                              // a candidate: X_q against its delta weights
+              ptx::tma_load_3d(a_dst, &tmXq, full_bar(stage), kb * BK16, mt * BM, 0);
+              ptx::tma_load_3d(a_dst + kABytes, &tmWq, full_bar(stage), kb * BK16, ot * BN, k);
             } else {
               ptx::tma_load_3d(a_dst, &tmXq, full_bar(stage), kb * BK8, mt * BM, k);
               ptx::tma_load_3d(a_dst + kABytes, &tmWq, full_bar(stage), kb * BK8, ot * BN, k);
@@ -161,7 +178,7 @@ gemm_w8a8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         for (int pass = 0; pass < passes && ok; ++pass, ++it) {
           const bool fp = !kApply && pass == 0;
-          const int nkb = fp ? args.num_kb16 : args.num_kb8;
+          const int nkb = fp ? (kDual ? 2 * args.num_kb16 : args.num_kb16) : (kDual ? args.num_kb16 : args.num_kb8);
           const int acc = (int)(it & 1);
           const uint32_t acc_phase = (uint32_t)((it >> 1) & 1);
           if (!ptx::mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) {
@@ -185,7 +202,9 @@ gemm_w8a8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             // four instructions per k-block either way: 16 bf16 or 32 int8 along K = 32 bytes per step
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks) {
-              if (fp) ptx::mma_bf16_ss(d_tmem, adesc + (uint64_t)(ks * 2), bdesc + (uint64_t)(ks * 2), kIdescBf16, accumulate);
+              if (fp || kDual)
+                ptx::mma_bf16_ss(d_tmem, adesc + (uint64_t)(ks * 2), bdesc + (uint64_t)(ks * 2),
+                                 (fp && kDual && kb >= args.num_kb16) ? kIdescBf16NegB : kIdescBf16, accumulate);
               else ptx::mma_i8_ss(d_tmem, adesc + (uint64_t)(ks * 2), bdesc + (uint64_t)(ks * 2), kIdescI8, accumulate);
               accumulate = 1;
             }
@@ -235,8 +254,8 @@ gemm_w8a8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
           continue;
         }
         const int k = kApply ? 0 : pass - 1;
-        const float tn = (n < n_tokens) ? args.t[(int64_t)k * args.N + n] : 0.0f;
-        const float* u_row = args.u + (int64_t)k * args.C2;
+        const float tn = (!kDual && n < n_tokens) ? args.t[(int64_t)k * args.N + n] : 0.0f;
+        const float* u_row = kDual ? nullptr : args.u + (int64_t)k * args.C2;
         if (!kApply) {
           float s0 = 0.f, s1 = 0.f;
 #pragma unroll
@@ -244,16 +263,24 @@ gemm_w8a8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             uint32_t r[8];
             ptx::tmem_ld8(taddr + c * 8, r);
             float tu[8];
+            if (!kDual) {
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              const int64_t col = col_base + c * 8 + j;
-              tu[j] = (col < args.C2) ? tn * __ldg(u_row + col) : 0.0f;
+              for (int j = 0; j < 8; ++j) {
+                const int64_t col = col_base + c * 8 + j;
+                tu[j] = (col < args.C2) ? tn * __ldg(u_row + col) : 0.0f;
+              }
             }
             ptx::tmem_ld_wait();
 #pragma unroll
             for (int j = 0; j < 8; j += 2) {
-              const float e0 = fmaf(-(float)(int)r[j], tu[j], yfp[c * 8 + j]);
-              const float e1 = fmaf(-(float)(int)r[j + 1], tu[j + 1], yfp[c * 8 + j + 1]);
+              float e0, e1;
+              if (kDual) {       // (X_fp - X_q) W^T + X_q dW_k^T, both fp32
+                e0 = yfp[c * 8 + j] + __uint_as_float(r[j]);
+                e1 = yfp[c * 8 + j + 1] + __uint_as_float(r[j + 1]);
+              } else {
+                e0 = fmaf(-(float)(int)r[j], tu[j], yfp[c * 8 + j]);
+                e1 = fmaf(-(float)(int)r[j + 1], tu[j + 1], yfp[c * 8 + j + 1]);
+              }
               s0 = fmaf(e0, e0, s0);
               s1 = fmaf(e1, e1, s1);
             }
@@ -325,11 +352,11 @@ int sm_count() {
   return sms;
 }
 
-template <bool kApply>
+template <int kMode>
 int configure_kernel() {
   static bool done = false;
   if (!done) {
-    TLQ_CUDA_TRY(cudaFuncSetAttribute(gemm_w8a8_kernel<kApply>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    TLQ_CUDA_TRY(cudaFuncSetAttribute(gemm_w8a8_kernel<kMode>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)kSmemBytes));
     done = true;
   }
@@ -369,7 +396,7 @@ int launch_search_gemm_i8(const uint16_t* X, const uint16_t* W, const int8_t* Xq
   if (!map_bf16_2d(&tmX, X, plan.N, plan.C1, BM) || !map_bf16_2d(&tmW, W, plan.C2, plan.C1, BN) ||
       !map_i8_3d(&tmXq, Xq, plan.N, plan.C1, plan.K, BM) || !map_i8_3d(&tmWq, Wq, plan.C2, plan.C1, plan.K, BN))
     return TLQ_ERR_CUDA;
-  int rc = configure_kernel<false>();
+  int rc = configure_kernel<0>();
   if (rc != TLQ_OK) return rc;
   I8Args a{};
   a.N = plan.N; a.C2 = plan.C2;
@@ -386,7 +413,7 @@ int launch_search_gemm_i8(const uint16_t* X, const uint16_t* W, const int8_t* Xq
   if (sms <= 0) return TLQ_ERR_CUDA;
   const unsigned grid = (unsigned)(a.num_tiles < sms ? a.num_tiles : sms);
   a.raster = make_raster(plan.mtiles, plan.otiles, sms, plan.N * plan.C1);
-  gemm_w8a8_kernel<false><<<grid, kThreads, kSmemBytes, st>>>(tmX, tmW, tmXq, tmWq, a);
+  gemm_w8a8_kernel<0><<<grid, kThreads, kSmemBytes, st>>>(tmX, tmW, tmXq, tmWq, a);
   return after_launch();
 }
 
@@ -394,7 +421,7 @@ int launch_apply_gemm_i8(const int8_t* Xq, const int8_t* Wq, const float* t, con
                          int64_t N, int64_t C1, int64_t C2, uint16_t* Yq, WorkspaceHeader* hdr, cudaStream_t st) {
   CUtensorMap tmXq, tmWq;
   if (!map_i8_3d(&tmXq, Xq, N, C1, 1, BM) || !map_i8_3d(&tmWq, Wq, C2, C1, 1, BN)) return TLQ_ERR_CUDA;
-  int rc = configure_kernel<true>();
+  int rc = configure_kernel<1>();
   if (rc != TLQ_OK) return rc;
   GemmPlan plan = plan_search_gemm_i8(N, C1, C2, 1);
   I8Args a{};
@@ -410,7 +437,43 @@ int launch_apply_gemm_i8(const int8_t* Xq, const int8_t* Wq, const float* t, con
   if (sms <= 0) return TLQ_ERR_CUDA;
   const unsigned grid = (unsigned)(a.num_tiles < sms ? a.num_tiles : sms);
   a.raster = make_raster(plan.mtiles, plan.otiles, sms, plan.N * plan.C1);
-  gemm_w8a8_kernel<true><<<grid, kThreads, kSmemBytes, st>>>(tmXq, tmWq, tmXq, tmWq, a);
+  gemm_w8a8_kernel<1><<<grid, kThreads, kSmemBytes, st>>>(tmXq, tmWq, tmXq, tmWq, a);
+  return after_launch();
+}
+
+// Two-stream search with 16-bit activations: partials / per-token layout as in the int8 search.
+int launch_search_gemm_dual_bf16(const uint16_t* Xq, const uint16_t* Xfp, const uint16_t* W, const uint16_t* dW,
+                                 const float* w_imp, const GemmPlan& plan, float* partials, float* ptab,
+                                 WorkspaceHeader* hdr, cudaStream_t st) {
+  CUtensorMap tmX, tmW, tmXq, tmD;
+  const uint64_t xdims[3] = {(uint64_t)plan.C1, (uint64_t)plan.N, 1};
+  const uint64_t xstr[2] = {(uint64_t)plan.C1 * 2, (uint64_t)plan.C1 * (uint64_t)plan.N * 2};
+  const uint32_t xbox[3] = {BK16, BM, 1};
+  const uint64_t ddims[3] = {(uint64_t)plan.C1, (uint64_t)plan.C2, (uint64_t)plan.K};
+  const uint64_t dstr[2] = {(uint64_t)plan.C1 * 2, (uint64_t)plan.C1 * (uint64_t)plan.C2 * 2};
+  const uint32_t dbox[3] = {BK16, BN, 1};
+  if (!map_bf16_2d(&tmX, Xfp, plan.N, plan.C1, BM) || !map_bf16_2d(&tmW, W, plan.C2, plan.C1, BN) ||
+      !encode_tensor_map(&tmXq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, Xq, xdims, xstr, xbox) ||
+      !encode_tensor_map(&tmD, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, dW, ddims, dstr, dbox))
+    return TLQ_ERR_CUDA;
+  int rc = configure_kernel<2>();
+  if (rc != TLQ_OK) return rc;
+  I8Args a{};
+  a.N = plan.N; a.C2 = plan.C2;
+  a.num_kb16 = (int)ceil_div(plan.C1, BK16);
+  a.num_kb8 = 0;
+  a.K = plan.K;
+  a.mtiles = plan.mtiles; a.otiles = plan.otiles;
+  a.num_tiles = plan.mtiles * plan.otiles;
+  a.n_pad = plan.n_pad;
+  a.w_imp = w_imp; a.t = nullptr; a.u = nullptr; a.partials = partials; a.ptab = ptab; a.bias = nullptr; a.yq = nullptr;
+  a.hdr = hdr;
+  a.n_live = nullptr;
+  const int sms = sm_count();
+  if (sms <= 0) return TLQ_ERR_CUDA;
+  const unsigned grid = (unsigned)(a.num_tiles < sms ? a.num_tiles : sms);
+  a.raster = make_raster(plan.mtiles, plan.otiles, sms, plan.N * plan.C1 * 2);
+  gemm_w8a8_kernel<2><<<grid, kThreads, kSmemBytes, st>>>(tmX, tmW, tmXq, tmD, a);
   return after_launch();
 }
 

@@ -29,7 +29,7 @@ STAGE_NAMES = ("stats", "fakequant", "gemm", "reduce")
 
 EXPORTS = (
     "tlq_status_string", "tlq_version", "tlq_token_importance", "tlq_scale_candidates_workspace_bytes",
-    "tlq_scale_candidates", "tlq_scale_candidates_noalloc", "tlq_quantize_weights", "tlq_quantize_activations", "tlq_scale_search_workspace_bytes", "tlq_scale_search_layer",
+    "tlq_scale_candidates", "tlq_scale_candidates_noalloc", "tlq_quantize_weights", "tlq_quantize_activations", "tlq_scale_search_workspace_bytes", "tlq_scale_search_layer", "tlq_scale_search_layer_two_stream",
     "tlq_apply_layer_workspace_bytes", "tlq_apply_layer", "tlq_read_status", "tlq_stage_timing_enable",
     "tlq_stage_timing_drain", "tlq_kernel_launch_count",
 )
@@ -83,6 +83,8 @@ def _load() -> ctypes.CDLL:
     lib.tlq_scale_search_workspace_bytes.restype = sz
     lib.tlq_scale_search_workspace_bytes.argtypes = [i64, i64, i64, cfgp]
     lib.tlq_scale_search_layer.argtypes = [vp, i64, i64, vp, i64, vp, vp, cfgp, vp, sz, vp, vp, vp, vp, vp]
+    lib.tlq_scale_search_layer_two_stream.argtypes = [vp, vp, i64, i64, vp, i64, vp, vp, cfgp, vp, sz, vp, vp, vp, vp, vp]
+    lib.tlq_scale_search_layer_two_stream.restype = i32
     lib.tlq_apply_layer_workspace_bytes.restype = sz
     lib.tlq_apply_layer_workspace_bytes.argtypes = [i64, i64, i64, cfgp]
     lib.tlq_apply_layer.argtypes = [vp, i64, i64, vp, i64, vp, vp, cfgp, vp, sz, vp, vp, vp, vp, vp]
@@ -210,17 +212,28 @@ class SearchBuffers:
 
 def tlq_scale_search_layer(X: torch.Tensor, W: torch.Tensor, w_imp: Optional[torch.Tensor], cfg: Config,
                            buffers: Optional[SearchBuffers] = None, mask: Optional[torch.Tensor] = None,
-                           per_token: bool = False, stream=None, check: bool = True) -> SearchBuffers:
-    """Enqueue the search; with check=True also synchronise and raise on a device-side error."""
+                           per_token: bool = False, stream=None, check: bool = True,
+                           X_fp: Optional[torch.Tensor] = None) -> SearchBuffers:
+    """Enqueue the search; with check=True also synchronise and raise on a device-side error.
+    X_fp selects tlq_scale_search_layer_two_stream (X is then the quantized stream)."""
     N, C1 = X.shape
     C2 = W.shape[0]
     if buffers is None:
         buffers = SearchBuffers(N, C1, C2, cfg, X.device, per_token)
     st = _stream(stream)
-    _check(lib.tlq_scale_search_layer(_ptr(X), N, C1, _ptr(W), C2, _ptr(w_imp), _ptr(mask), ctypes.byref(cfg),
-                                      _ptr(buffers.workspace), buffers.nbytes, _ptr(buffers.best_idx),
-                                      _ptr(buffers.losses), _ptr(buffers.s_best), _ptr(buffers.per_token), st),
-           "tlq_scale_search_layer")
+    if X_fp is None:
+        _check(lib.tlq_scale_search_layer(_ptr(X), N, C1, _ptr(W), C2, _ptr(w_imp), _ptr(mask), ctypes.byref(cfg),
+                                          _ptr(buffers.workspace), buffers.nbytes, _ptr(buffers.best_idx),
+                                          _ptr(buffers.losses), _ptr(buffers.s_best), _ptr(buffers.per_token), st),
+               "tlq_scale_search_layer")
+    else:
+        if X_fp.shape != X.shape:
+            raise ValueError("X_fp must have the shape of X")
+        _check(lib.tlq_scale_search_layer_two_stream(_ptr(X), _ptr(X_fp), N, C1, _ptr(W), C2, _ptr(w_imp), _ptr(mask),
+                                                     ctypes.byref(cfg), _ptr(buffers.workspace), buffers.nbytes,
+                                                     _ptr(buffers.best_idx), _ptr(buffers.losses), _ptr(buffers.s_best),
+                                                     _ptr(buffers.per_token), st),
+               "tlq_scale_search_layer_two_stream")
     if check:
         _check(lib.tlq_read_status(_ptr(buffers.workspace), st), "tlq_scale_search_layer (device)")
     return buffers

@@ -54,7 +54,9 @@ def test_workspace_queries_and_shape_validation(tlq):
     assert tlq.tlq_scale_search_workspace_bytes(0, 512, 512, c) == 0
     bad = tlq.config(n_grid=65)
     assert tlq.tlq_scale_search_workspace_bytes(256, 512, 512, bad) == 0
-    assert tlq.lib.tlq_scale_candidates_workspace_bytes(8192, 3584) >= 128 * 3584 * 8
+    # fp64 column partials: one row of C1 doubles per chunk of 256 tokens
+    assert tlq.lib.tlq_scale_candidates_workspace_bytes(8192, 3584) == 32 * 3584 * 8
+    assert tlq.lib.tlq_scale_candidates_workspace_bytes(1, 8) == 256
 
 
 @pytest.mark.skipif(torch.cuda.is_available(), reason="checks the no-device error path")

@@ -491,3 +491,51 @@ def test_search_on_cta_pairs(tlq, n, c1, c2, group, n_grid):
     cfg2 = tlq.config(group_size=group, n_grid=n_grid, flags=tlq.FLAG_GEMM_CTA_PAIRS | tlq.FLAG_SKIP_ZERO_WEIGHT_TOKENS)
     out2 = tlq.tlq_scale_search_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), torch.from_numpy(imp2).cuda(), cfg2)
     np.testing.assert_allclose(out2.losses.cpu().numpy(), ref2["losses"], rtol=LOSS_RTOL)
+
+
+# ----------------------------------------------------------------------------------- two activation streams
+
+
+def _perturbed_stream(xb, seed, rel):
+    """A second activation stream: the same tokens with a relative perturbation (what the quantized layers
+    before this one would have done to them), rounded to bf16."""
+    x = wl.bf16_bits_to_f32(xb)
+    noise = np.random.default_rng(seed).standard_normal(x.shape).astype(np.float32)
+    return wl.f32_to_bf16_bits(x * (1.0 + rel * noise))
+
+
+@pytest.mark.parametrize("mode", ["w4a16", "w8a8", "w4a8"])
+@pytest.mark.parametrize("n,c1,c2,n_grid,rel", [(256, 512, 512, 20, 0.02), (300, 288, 320, 5, 0.1), (130, 128, 100, 3, 0.5),
+                                                (515, 1088, 777, 6, 0.02), (1, 64, 8, 2, 0.1)])
+def test_two_stream_search(tlq, mode, n, c1, c2, n_grid, rel):
+    """First propagation strategy of Sec. 3.2.1: reference output from x_fp, quantized layer (and scale) from x_q."""
+    xf, wb, imp = wl.small_case(121, n, c1, c2)
+    xq = _perturbed_stream(xf, 7, rel)
+    if mode == "w4a16":
+        cfg = tlq.config(group_size=32, n_grid=n_grid)
+        ref = orc.scale_search(xq, wb, imp, "w4a16", 32, n_grid, x_fp_bits=xf)
+    else:
+        wn, an = orc.symmetric_bits(mode)
+        cfg = tlq.config(tlq.WA_SYM_CHANNEL, w_bits=wn, a_bits=an, n_grid=n_grid)
+        ref = orc.scale_search(xq, wb, imp, mode, 0, n_grid, x_fp_bits=xf)
+    out = tlq.tlq_scale_search_layer(dev_bf16(tlq, xq), dev_bf16(tlq, wb), torch.from_numpy(imp).cuda(), cfg,
+                                     per_token=True, X_fp=dev_bf16(tlq, xf))
+    got = dict(best=int(out.best_idx.item()), losses=out.losses.cpu().numpy(), per_token=out.per_token.cpu().numpy(),
+               s_best=bits_of(out.s_best))
+    check_against_oracle(got, ref, n_grid)
+
+
+def test_two_stream_with_equal_streams_is_the_plain_search(tlq):
+    xb, wb, imp = wl.small_case(123, 384, 256, 320)
+    cfg = tlq.config(group_size=64, n_grid=6)
+    w_dev = torch.from_numpy(imp).cuda()
+    one = tlq.tlq_scale_search_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), w_dev, cfg, per_token=True)
+    two = tlq.tlq_scale_search_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), w_dev, cfg, per_token=True, X_fp=dev_bf16(tlq, xb))
+    assert int(one.best_idx.item()) == int(two.best_idx.item())
+    # X W^T - X W^T cancels exactly in the fp32 accumulator, what remains is the same X dW^T
+    np.testing.assert_allclose(two.per_token.cpu().numpy(), one.per_token.cpu().numpy(), rtol=1e-5)
+    with pytest.raises(tlq.TlqError) as e:
+        tlq.tlq_scale_search_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), w_dev,
+                                   tlq.config(group_size=64, n_grid=6, flags=tlq.FLAG_SKIP_ZERO_WEIGHT_TOKENS),
+                                   X_fp=dev_bf16(tlq, xb))
+    assert e.value.status == tlq.ERR_INVALID_ARG
