@@ -11,7 +11,7 @@ from __future__ import annotations
 
 import dataclasses
 import os
-from typing import List, Optional, Sequence
+from typing import List, Optional, Sequence, Tuple
 
 import torch
 import torch.distributed as dist
@@ -68,3 +68,34 @@ def max_over_ranks(values: Sequence[float], info: RankInfo, device: Optional[tor
 def whole_job_rate(units_per_rank_step: float, steps: int, info: RankInfo, max_ms: float) -> float:
     """Units all ranks processed per second, given the max-over-ranks time of `steps` steps."""
     return info.world * units_per_rank_step * steps / (max_ms * 1e-3)
+
+
+# ----------------------------------------------------------------------------- one layer sharded over ranks
+# Quantizers act per output row (or per group inside a row), so a weight matrix can be cut by rows: every
+# rank searches its slice of W against the same tokens and the K slice losses combine exactly, weighted
+# by the row counts.  The only exchange is one SUM reduction of K doubles; every rank then takes the
+# same argmin.
+
+
+def shard_rows(c_out: int, info: RankInfo) -> Tuple[int, int]:
+    """[row0, row1) of this rank: contiguous, sizes differing by at most one row."""
+    base, extra = divmod(int(c_out), info.world)
+    row0 = info.rank * base + min(info.rank, extra)
+    return row0, row0 + base + (1 if info.rank < extra else 0)
+
+
+def combine_sharded_losses(local_losses: torch.Tensor, local_rows: int, c_out: int, info: RankInfo):
+    """Losses of the whole matrix from the ranks' slice losses (each normalised by its own row count, as the
+    search returns them): sum_r rows_r * loss_r / c_out.  Returns (losses float64 [K], argmin with the lowest
+    index on ties).  `local_losses` may live on the GPU (NCCL) or the CPU (gloo)."""
+    t = local_losses.to(torch.float64) * float(local_rows)
+    if info.world > 1:
+        t = t.clone()
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    total = t / float(c_out)
+    vals = total.cpu().tolist()
+    best, bv = 0, float("inf")
+    for k, v in enumerate(vals):
+        if v < bv:
+            best, bv = k, v
+    return total, best

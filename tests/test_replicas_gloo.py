@@ -62,6 +62,38 @@ def _worker(rank: int, world: int, port: int, out_dir: str) -> None:
         dist.destroy_process_group()
 
 
+def _shard_worker(rank: int, world: int, port: int, out_dir: str) -> None:
+    """One linear cut by output rows over the ranks: slice losses from the oracle, combined over gloo."""
+    sys.path.insert(0, ROOT)
+    from oracle import tlq_oracle as orc
+    from paper_2602_07899_b200 import replicas, workloads as wl
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world),
+                      LOCAL_RANK=str(rank))
+    info = replicas.rank_info_from_env()
+    replicas.init_process_group(info, "gloo")
+    try:
+        x, w, imp = wl.small_case(131, 48, 64, 37)           # 37 rows: uneven slices
+        r0, r1 = replicas.shard_rows(37, info)
+        spans = [None] * world
+        dist.all_gather_object(spans, (r0, r1))
+        assert spans[0][0] == 0 and spans[-1][1] == 37 and all(spans[i][1] == spans[i + 1][0] for i in range(world - 1))
+        for mode, group in (("w4a16", 32), ("w4a8", 0)):
+            mine = orc.scale_search(x, w[r0:r1], imp, mode=mode, group=group, n_grid=5)
+            total, best = replicas.combine_sharded_losses(torch.from_numpy(mine["losses"]), r1 - r0, 37, info)
+            full = orc.scale_search(x, w, imp, mode=mode, group=group, n_grid=5)
+            assert np.allclose(total.numpy(), full["losses"], rtol=1e-12)
+            assert best == full["best"]
+        with open(os.path.join(out_dir, f"shard{rank}"), "w") as f:
+            f.write("ok")
+    finally:
+        dist.destroy_process_group()
+
+
+def test_row_sharded_search_combines_exactly(tmp_path):
+    mp.spawn(_shard_worker, args=(2, _free_port(), str(tmp_path)), nprocs=2, join=True)
+    assert sorted(os.listdir(tmp_path)) == ["shard0", "shard1"]
+
+
 def test_two_gloo_ranks_host_logic(tmp_path):
     port = _free_port()
     mp.spawn(_worker, args=(2, port, str(tmp_path)), nprocs=2, join=True)
