@@ -221,6 +221,7 @@ def run_ours(args, cfgw):
     data = wl.LayerData(cfgr)
     lins = [l for l in cfgr.linears() if args.linears is None or l.name in args.linears.split(",")]
     flags = tlq.FLAG_SKIP_ZERO_WEIGHT_TOKENS if args.skip_zero_weight else 0
+    flags |= {"default": 0, "pairs": tlq.FLAG_GEMM_CTA_PAIRS, "narrow": tlq.FLAG_GEMM_NARROW_TILES}[args.gemm]
     if cfgr.mode == "w4a16":
         cfg = tlq.config(mode=tlq.W4A16_ASYM_GROUP, group_size=cfgr.group, n_grid=cfgr.n_grid, flags=flags)
     else:   # "w<n>a<m>": symmetric per-channel weights / per-token activations on the int8 tensor-core path
@@ -357,7 +358,8 @@ def run_ours(args, cfgw):
     achieved = gemm_flops_sum / (gemm_ms_sum * 1e-3) / 1e12 if gemm_ms_sum > 0 else None
     traffic = None
     tpath = os.path.join(ROOT, "profiles", "search_gemm_traffic.json")
-    if os.path.exists(tpath) and args.linears is None and args.mode is None and not args.skip_zero_weight:
+    if os.path.exists(tpath) and args.linears is None and args.mode is None and not args.skip_zero_weight \
+            and args.gemm == "default":
         with open(tpath) as f:      # ncu counters of this very workload and kernel; anything else has none
             traffic = json.load(f).get(cfgr.key)
     i8 = cfgr.mode != "w4a16"
@@ -366,7 +368,7 @@ def run_ours(args, cfgw):
     ratio = 2.0 if i8 else 1.0
     peak = peaks["bf16_sustained"] * ratio
     nominal = 2250.0 * ratio
-    roofline = {"kernel": "gemm_w8a8_kernel<search>" if i8 else "gemm_bf16_kernel<search>", "bound": "tensor",
+    roofline = {"kernel": "gemm_w8a8_kernel<search>" if i8 else {"default": "gemm_bf16_wide_kernel", "pairs": "gemm_bf16_pair_kernel", "narrow": "gemm_bf16_kernel<search>"}[args.gemm], "bound": "tensor",
                 "achieved": achieved, "peak": peak, "unit": "TOP/s" if i8 else "TFLOP/s",
                 "frac": (achieved / peak) if achieved else None, "traffic": traffic,
                 "peak_source": (f"{peaks['source']} (sustained cuBLAS bf16 {peaks['bf16_sustained']}"
@@ -413,6 +415,8 @@ def main():
                     help="token weights: the config's (log-normal) or a 0/1 top-50%% mask (the paper's token set)")
     ap.add_argument("--skip-zero-weight", action="store_true",
                     help="set TLQ_FLAG_SKIP_ZERO_WEIGHT_TOKENS (tensor FLOP/s then count the live tokens only)")
+    ap.add_argument("--gemm", default="default", choices=["default", "pairs", "narrow"],
+                    help="variant of the bf16 search GEMM (TLQ_FLAG_GEMM_*), for A/B measurements")
     ap.add_argument("--linears", default=None, help="comma-separated subset of q,k,v,o,gate,up,down (profiling)")
     ap.add_argument("--profile", action="store_true", help="kernel leg only: skip the end-to-end and CPU legs")
     args = ap.parse_args()

@@ -79,6 +79,11 @@ extern "C" {
                                                Off by default: equal speed in isolation, slower under the power cap
                                                of a long run on the parts measured. */
 
+#define TLQ_FLAG_GEMM_NARROW_TILES 4u       /* tlq_scale_search_layer, group mode: one CTA per 128-token x 256-channel
+                                               tile, as used for N <= 128, instead of the default 256-token tile that
+                                               stages the weight tile once for two 128-token halves (measured 8 %
+                                               faster inside a benchmark step). */
+
 #define TLQ_MAX_GRID 64
 
 typedef struct {

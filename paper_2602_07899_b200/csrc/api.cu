@@ -15,7 +15,7 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 int check_cfg(const tlq_config* cfg, int64_t C1, bool need_quantizer = true) {
   if (cfg == nullptr || cfg->struct_size != sizeof(tlq_config)) return TLQ_ERR_INVALID_ARG;
-  if ((cfg->flags & ~(uint32_t)(TLQ_FLAG_SKIP_ZERO_WEIGHT_TOKENS | TLQ_FLAG_GEMM_CTA_PAIRS)) != 0)
+  if ((cfg->flags & ~(uint32_t)(TLQ_FLAG_SKIP_ZERO_WEIGHT_TOKENS | TLQ_FLAG_GEMM_CTA_PAIRS | TLQ_FLAG_GEMM_NARROW_TILES)) != 0)
     return TLQ_ERR_INVALID_ARG;
   if (cfg->n_grid < 1 || cfg->n_grid > TLQ_MAX_GRID) return TLQ_ERR_SHAPE;
   if (cfg->stat_mode < TLQ_STAT_MEAN_ABS || cfg->stat_mode > TLQ_STAT_MASKED_MAX) return TLQ_ERR_INVALID_ARG;
@@ -285,7 +285,8 @@ static int search_impl(const void* X, const void* X_ref, int64_t N, int64_t C1, 
   const bool compact = (cfg->flags & TLQ_FLAG_SKIP_ZERO_WEIGHT_TOKENS) != 0;
   if (compact && (w_imp == nullptr || per_token_err != nullptr)) return TLQ_ERR_INVALID_ARG;
   const bool two_stream = X_ref != nullptr;
-  if (two_stream && (cfg->flags & (TLQ_FLAG_SKIP_ZERO_WEIGHT_TOKENS | TLQ_FLAG_GEMM_CTA_PAIRS)) != 0)
+  if (two_stream &&
+      (cfg->flags & (TLQ_FLAG_SKIP_ZERO_WEIGHT_TOKENS | TLQ_FLAG_GEMM_CTA_PAIRS | TLQ_FLAG_GEMM_NARROW_TILES)) != 0)
     return TLQ_ERR_INVALID_ARG;
   if (!aligned16(X) || !aligned16(W) || !aligned16(workspace) || !aligned16(X_ref)) return TLQ_ERR_ALIGN;
   SearchLayout L = carve_search(workspace, N, C1, C2, cfg);
@@ -327,7 +328,9 @@ static int search_impl(const void* X, const void* X_ref, int64_t N, int64_t C1, 
     } else if (cfg->flags & TLQ_FLAG_GEMM_CTA_PAIRS) {
       if ((rc = launch_search_gemm_bf16_pair(Xg, L.dW, wg, L.plan, L.partials, ptab, L.hdr, n_live, st)) != TLQ_OK)
         return rc;
-    } else if ((rc = launch_search_gemm_bf16(Xg, L.dW, wg, L.plan, L.partials, ptab, L.hdr, n_live, st)) != TLQ_OK) {
+    } else if ((cfg->flags & TLQ_FLAG_GEMM_NARROW_TILES) || N <= 128) {
+      if ((rc = launch_search_gemm_bf16(Xg, L.dW, wg, L.plan, L.partials, ptab, L.hdr, n_live, st)) != TLQ_OK) return rc;
+    } else if ((rc = launch_search_gemm_bf16_wide(Xg, L.dW, wg, L.plan, L.partials, ptab, L.hdr, n_live, st)) != TLQ_OK) {
       return rc;
     }
   } else {

@@ -173,6 +173,10 @@ int search_gemm_pair_capacity();
 int launch_search_gemm_bf16_pair(const uint16_t* X, const uint16_t* dW, const float* w_imp, const GemmPlan& plan,
                                  float* partials, float* ptab, WorkspaceHeader* hdr, const int32_t* n_live,
                                  cudaStream_t st);
+// search_gemm_wide.cu: the same search on 256-token x 256-channel tiles per CTA (weight tile shared by two halves)
+int launch_search_gemm_bf16_wide(const uint16_t* X, const uint16_t* dW, const float* w_imp, const GemmPlan& plan,
+                                 float* partials, float* ptab, WorkspaceHeader* hdr, const int32_t* n_live,
+                                 cudaStream_t st);
 // Apply: Yq[N,C2] = X W^T - X dW^T (+bias), bf16 out
 int launch_apply_gemm_bf16(const uint16_t* X, const uint16_t* W, const uint16_t* dW, const uint16_t* bias,
                            int64_t N, int64_t C1, int64_t C2, uint16_t* Yq, WorkspaceHeader* hdr, cudaStream_t st);

@@ -472,12 +472,15 @@ def test_skipping_needs_weights_and_has_no_per_token_table(tlq):
 
 @pytest.mark.parametrize("n,c1,c2,group,n_grid", [(256, 512, 512, 128, 20), (300, 288, 320, 32, 5), (130, 128, 100, 64, 3),
                                                   (1, 64, 8, 32, 2), (515, 1088, 777, 64, 6), (1000, 512, 256, 128, 4)])
-def test_search_on_cta_pairs(tlq, n, c1, c2, group, n_grid):
-    """The same search with the fused GEMM on CTA pairs (256-token tiles across two SMs): oracle parity, and the
-    odd-tile and ragged cases where the second CTA of a pair has no tokens."""
+@pytest.mark.parametrize("variant", ["pairs", "narrow"])
+def test_search_on_cta_pairs(tlq, n, c1, c2, group, n_grid, variant):
+    """The search with the other variants of the fused GEMM (the default is one CTA per 256-token tile): 256-token
+    tiles across two SMs (CTA pairs) and 128-token tiles; oracle parity, including the odd-tile and ragged cases
+    where the second half of a 256-token tile has no tokens."""
+    gemm_flag = tlq.FLAG_GEMM_CTA_PAIRS if variant == "pairs" else tlq.FLAG_GEMM_NARROW_TILES
     xb, wb, imp = wl.small_case(101, n, c1, c2)
     ref = orc.scale_search(xb, wb, imp, "w4a16", group, n_grid)
-    cfg = tlq.config(group_size=group, n_grid=n_grid, flags=tlq.FLAG_GEMM_CTA_PAIRS)
+    cfg = tlq.config(group_size=group, n_grid=n_grid, flags=gemm_flag)
     out = tlq.tlq_scale_search_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), torch.from_numpy(imp).cuda(), cfg, per_token=True)
     got = dict(best=int(out.best_idx.item()), losses=out.losses.cpu().numpy(), per_token=out.per_token.cpu().numpy(),
                s_best=bits_of(out.s_best))
@@ -488,7 +491,7 @@ def test_search_on_cta_pairs(tlq, n, c1, c2, group, n_grid):
     if imp2.sum() == 0.0:
         return
     ref2 = orc.scale_search(xb, wb, imp2, "w4a16", group, n_grid)
-    cfg2 = tlq.config(group_size=group, n_grid=n_grid, flags=tlq.FLAG_GEMM_CTA_PAIRS | tlq.FLAG_SKIP_ZERO_WEIGHT_TOKENS)
+    cfg2 = tlq.config(group_size=group, n_grid=n_grid, flags=gemm_flag | tlq.FLAG_SKIP_ZERO_WEIGHT_TOKENS)
     out2 = tlq.tlq_scale_search_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), torch.from_numpy(imp2).cuda(), cfg2)
     np.testing.assert_allclose(out2.losses.cpu().numpy(), ref2["losses"], rtol=LOSS_RTOL)
 
