@@ -542,3 +542,26 @@ def test_two_stream_with_equal_streams_is_the_plain_search(tlq):
                                    tlq.config(group_size=64, n_grid=6, flags=tlq.FLAG_SKIP_ZERO_WEIGHT_TOKENS),
                                    X_fp=dev_bf16(tlq, xb))
     assert e.value.status == tlq.ERR_INVALID_ARG
+
+
+# ----------------------------------------------------------------------------------- grid extremes
+
+
+@pytest.mark.parametrize("mode", ["w4a16", "w8a8"])
+@pytest.mark.parametrize("n_grid", [1, 64])
+def test_grid_of_one_and_of_the_maximum(tlq, mode, n_grid):
+    """K = 1 (only scale = 1, plain round-to-nearest) and K = 64 (TLQ_MAX_GRID); K = 65 is refused."""
+    xb, wb, imp = wl.small_case(141, 200, 128, 96)
+    if mode == "w4a16":
+        cfg = tlq.config(group_size=64, n_grid=n_grid)
+        ref = orc.scale_search(xb, wb, imp, "w4a16", 64, n_grid)
+    else:
+        cfg = tlq.config(tlq.W8A8_SYM, n_grid=n_grid)
+        ref = orc.scale_search(xb, wb, imp, "w8a8", 0, n_grid)
+    out = tlq.tlq_scale_search_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), torch.from_numpy(imp).cuda(), cfg, per_token=True)
+    got = dict(best=int(out.best_idx.item()), losses=out.losses.cpu().numpy(), per_token=out.per_token.cpu().numpy(),
+               s_best=bits_of(out.s_best))
+    check_against_oracle(got, ref, n_grid)
+    if n_grid == 1:
+        assert got["best"] == 0 and np.all(wl.bf16_bits_to_f32(got["s_best"]) == 1.0)
+    assert tlq.tlq_scale_search_workspace_bytes(200, 128, 96, tlq.config(n_grid=65)) == 0
