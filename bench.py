@@ -29,9 +29,10 @@ import numpy as np  # noqa: E402
 
 METRIC = "scale_grid_candidates_per_sec"
 UNIT = "candidates/s"
-SAMPLE_LINEAR = "k"
-SAMPLE_TOKENS = 2048           # per step of the reference arm (many steps: keep each near a second)
-BASELINE_TOKENS = 16384        # the one-shot cpu_baseline leg of the GPU arm (about 5-20 s of CPU work)
+SAMPLE_LINEAR = "k"            # reference arm: k-projection, first SAMPLE_TOKENS tokens per step (about a second)
+SAMPLE_TOKENS = 2048
+BASELINE_LINEAR = "q"          # the one-shot cpu_baseline leg of the GPU arm: q-projection, first BASELINE_TOKENS
+BASELINE_TOKENS = 4096         # tokens (about 10-25 s of CPU work on 16 cores)
 
 
 def measured_peaks():
@@ -51,11 +52,11 @@ def layer_flops(cfgw):
 # --------------------------------------------------------------------------------------------- CPU oracle legs
 
 
-def oracle_sample_seconds(cfgw, data, tokens=SAMPLE_TOKENS):
+def oracle_sample_seconds(cfgw, data, tokens=SAMPLE_TOKENS, linear=SAMPLE_LINEAR):
     """One pass of the oracle over the bounded sample: one projection, the first `tokens` tokens,
     all K candidates.  Returns (seconds, flops of the sample)."""
     from oracle import tlq_oracle as orc
-    lin = cfgw.linear(SAMPLE_LINEAR)
+    lin = cfgw.linear(linear)
     n = min(tokens, cfgw.n_tokens)
     x, w, imp = data.x(lin)[:n], data.w(lin), data.imp()[:n]
     t0 = time.perf_counter()
@@ -64,10 +65,10 @@ def oracle_sample_seconds(cfgw, data, tokens=SAMPLE_TOKENS):
     return dt, 2.0 * n * lin.c_in * lin.c_out * cfgw.n_grid
 
 
-def sample_description(cfgw, tokens=SAMPLE_TOKENS):
-    lin = cfgw.linear(SAMPLE_LINEAR)
+def sample_description(cfgw, tokens=SAMPLE_TOKENS, linear=SAMPLE_LINEAR):
+    lin = cfgw.linear(linear)
     n = min(tokens, cfgw.n_tokens)
-    return (f"{SAMPLE_LINEAR}-projection {lin.c_in}->{lin.c_out}, first {n} of {cfgw.n_tokens} tokens, all "
+    return (f"{linear}-projection {lin.c_in}->{lin.c_out}, first {n} of {cfgw.n_tokens} tokens, all "
             f"{cfgw.n_grid} candidates; scaled to the whole layer by 2*N*C1*C2*K (extrapolated)")
 
 
@@ -384,9 +385,9 @@ def run_ours(args, cfgw):
 
     cpu = None
     if world == 1:
-        dt, fl = oracle_sample_seconds(cfgw, data, BASELINE_TOKENS)
+        dt, fl = oracle_sample_seconds(cfgw, data, BASELINE_TOKENS, BASELINE_LINEAR)
         cpu = {"value": candidates_per_sec_from_sample(cfgw, dt, fl), "unit": UNIT, "cores": os.cpu_count(),
-               "kind": "oracle", "sample": sample_description(cfgw, BASELINE_TOKENS), "sample_seconds": round(dt, 3),
+               "kind": "oracle", "sample": sample_description(cfgw, BASELINE_TOKENS, BASELINE_LINEAR), "sample_seconds": round(dt, 3),
                "oracle_gflops": round(fl / dt / 1e9, 1)}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
