@@ -90,6 +90,24 @@ def test_host_validation_error_codes(tlq):
     cm = tlq.config(stat_mode=tlq.STAT_MASKED_MAX)
     assert L.tlq_scale_search_layer(a, 4, 128, a, 8, None, None, ctypes.byref(cm), a, 1 << 30, a, a, a, None,
                                     None) == tlq.ERR_INVALID_ARG
+    # flags: unknown bits, token skipping without weights or with a per-token table, options the two-stream call rejects
+    assert L.tlq_scale_search_layer(a, 4, 128, a, 8, None, None, ctypes.byref(tlq.config(flags=8)), a, 1 << 30, a, a, a,
+                                    None, None) == tlq.ERR_INVALID_ARG
+    skip = tlq.config(flags=tlq.FLAG_SKIP_ZERO_WEIGHT_TOKENS)
+    assert L.tlq_scale_search_layer(a, 4, 128, a, 8, None, None, ctypes.byref(skip), a, 1 << 30, a, a, a, None,
+                                    None) == tlq.ERR_INVALID_ARG
+    assert L.tlq_scale_search_layer(a, 4, 128, a, 8, a, None, ctypes.byref(skip), a, 1 << 30, a, a, a, a,
+                                    None) == tlq.ERR_INVALID_ARG
+    assert L.tlq_scale_search_layer_two_stream(a, None, 4, 128, a, 8, None, None, ctypes.byref(c), a, 1 << 30, a, a, a,
+                                               None, None) == tlq.ERR_INVALID_ARG
+    assert L.tlq_scale_search_layer_two_stream(a, a, 4, 128, a, 8, a, None, ctypes.byref(skip), a, 1 << 30, a, a, a,
+                                               None, None) == tlq.ERR_INVALID_ARG
+    assert L.tlq_scale_search_layer_two_stream(a, a + 4, 4, 128, a, 8, None, None, ctypes.byref(c), a, 1 << 30, a, a, a,
+                                               None, None) == tlq.ERR_ALIGN
+    # the symmetric mode takes 2..8 bits on either side, nothing else
+    assert tlq.tlq_scale_search_workspace_bytes(64, 128, 64, tlq.config(tlq.WA_SYM_CHANNEL, w_bits=4, a_bits=6)) > 0
+    assert tlq.tlq_scale_search_workspace_bytes(64, 128, 64, tlq.config(tlq.WA_SYM_CHANNEL, w_bits=4, a_bits=16)) == 0
+    assert tlq.tlq_scale_search_workspace_bytes(64, 128, 64, tlq.config(tlq.WA_SYM_CHANNEL, w_bits=1, a_bits=8)) == 0
     assert L.tlq_token_importance(a, 7, 1, 4, 8, 0, 0.0, a, None, None) == tlq.ERR_INVALID_ARG
     assert L.tlq_token_importance(a, 0, 1, 4, 12, 0, 0.0, a, None, None) == tlq.ERR_SHAPE
     assert L.tlq_token_importance(a, 0, 1, 4, 8, 0, 1.5, a, None, None) == tlq.ERR_INVALID_ARG
