@@ -164,6 +164,16 @@ int tlq_quantize_weights(const void* W, const void* s, int64_t C2, int64_t C1, c
                          uint8_t* codes, float* steps, int32_t* zeros, void* dW_out, void* stream);
 
 /*
+ * Storage format for 4-bit weights (Sec. 2.2, integer range for n = 4: sixteen levels, half a byte per weight):
+ * packs the one-code-per-byte output of tlq_quantize_weights / tlq_apply_layer two per byte,
+ *   packed[r, j] = (codes[r, 2j] & 15) | (codes[r, 2j+1] & 15) << 4,
+ * for the group mode's unsigned codes (0..15) as well as the symmetric mode's integers (-8..7, which stay
+ * two's-complement nibbles).  codes [rows, cols] one per byte, cols a multiple of 32; packed [rows, cols/2].
+ * Only the low four bits of every code are kept: the caller quantized with w_bits <= 4.
+ */
+int tlq_pack_codes4(const uint8_t* codes, int64_t rows, int64_t cols, uint8_t* packed, void* stream);
+
+/*
  * Quantize the smoothed activations for ONE scale vector: Q_a(x / scale), per-token symmetric, a_bits wide
  * (Sec. 2.2 first two equations; Sec. 3.2.1 f_q).  Symmetric mode only.
  *   X [N,C1] bf16; s [C1] bf16 or NULL (= ones); codes [N,C1] int8; steps [N] fp32.

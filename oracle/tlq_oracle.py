@@ -191,6 +191,22 @@ def quantize_activations_token_sym(x_bits: np.ndarray, s: np.ndarray | None, bit
     return quantize_sym_rows(xt, bits)
 
 
+def pack_codes4(codes: np.ndarray) -> np.ndarray:
+    """Two 4-bit codes per byte, the even channel in the low nibble (a storage format: with n = 4 the
+    integer range of Sec. 2.2 has sixteen levels).  Signed codes keep their two's-complement nibble."""
+    c = np.asarray(codes).astype(np.int64) & 15
+    return (c[:, 0::2] | (c[:, 1::2] << 4)).astype(np.uint8)
+
+
+def unpack_codes4(packed: np.ndarray, signed: bool) -> np.ndarray:
+    """Inverse of pack_codes4: [R,C/2] bytes -> [R,C] integers in 0..15, or -8..7 when `signed`."""
+    p = np.asarray(packed, dtype=np.uint8).astype(np.int64)
+    out = np.empty((p.shape[0], 2 * p.shape[1]), dtype=np.int64)
+    out[:, 0::2] = p & 15
+    out[:, 1::2] = p >> 4
+    return np.where(out >= 8, out - 16, out) if signed else out
+
+
 # ----------------------------------------------------------------------------- the layer, its error, the search
 
 

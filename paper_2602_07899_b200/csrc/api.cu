@@ -248,6 +248,15 @@ int tlq_quantize_weights(const void* W, const void* s, int64_t C2, int64_t C1, c
   return launch_fakequant_rows_i8(Wb, sb, 1, C2, C1, cfg->w_bits, reinterpret_cast<int8_t*>(codes), steps, st);
 }
 
+int tlq_pack_codes4(const uint8_t* codes, int64_t rows, int64_t cols, uint8_t* packed, void* stream) {
+  if (codes == nullptr || packed == nullptr) return TLQ_ERR_INVALID_ARG;
+  if (rows < 1 || cols < 32 || (cols % 32) != 0) return TLQ_ERR_SHAPE;
+  if (!aligned16(codes) || !aligned16(packed)) return TLQ_ERR_ALIGN;
+  int rc = have_device();
+  if (rc != TLQ_OK) return rc;
+  return launch_pack_codes4(codes, rows * cols, packed, reinterpret_cast<cudaStream_t>(stream));
+}
+
 int tlq_quantize_activations(const void* X, const void* s, int64_t N, int64_t C1, const tlq_config* cfg, int8_t* codes,
                              float* steps, void* stream) {
   if (X == nullptr || codes == nullptr || steps == nullptr) return TLQ_ERR_INVALID_ARG;

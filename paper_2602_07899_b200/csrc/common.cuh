@@ -143,6 +143,9 @@ int launch_actquant_i8(const uint16_t* X, const uint16_t* s, const float* rs, in
 int launch_compact_tokens(const uint16_t* X, const float* w_imp, int64_t N, int64_t n_pad, int64_t C1, int32_t* idx,
                           float* wc, int32_t* live, uint16_t* Xc, cudaStream_t st);
 
+// 4-bit codes, two per byte (even channel in the low nibble); n_codes a multiple of 32
+int launch_pack_codes4(const uint8_t* codes, int64_t n_codes, uint8_t* packed, cudaStream_t st);
+
 // importance.cu
 int launch_token_importance(const void* G, int g_dtype, int64_t B, int64_t N, int64_t C, int norm_kind,
                             float* imp, cudaStream_t st);

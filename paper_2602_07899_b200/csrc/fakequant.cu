@@ -674,4 +674,29 @@ int launch_actquant_i8(const uint16_t* X, const uint16_t* s, const float* rs, in
   return launch_rows<kMultRecipOfScale>(X, s, nullptr, K, N, C1, bits, q, t, n_rows_dev, st);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Storage format of 4-bit codes: two per byte, the even channel in the low nibble.  Works for the
+// unsigned codes of the group mode (0..15) and for the symmetric mode's integers (-8..7, kept as
+// two's-complement nibbles).  One thread packs 32 codes (two 128-bit loads, one 128-bit store).
+// ------------------------------------------------------------------------------------------------
+__global__ void pack_codes4_kernel(const uint8_t* __restrict__ codes, int64_t n_packets, uint8_t* __restrict__ packed) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;      // packet of 32 codes -> 16 bytes
+  if (i >= n_packets) return;
+  const uint4 a = ld_nc_16(codes + i * 32), b = ld_nc_16(codes + i * 32 + 16);
+  auto pack8 = [](uint32_t lo, uint32_t hi) {     // 8 codes (one per byte in lo, hi) -> 4 bytes
+    const uint32_t l = lo & 0x0F0F0F0Fu, h = hi & 0x0F0F0F0Fu;
+    const uint32_t pl = (l | (l >> 4)) & 0x00FF00FFu;        // bytes 0 and 2 hold the pairs (c0,c1) and (c2,c3)
+    const uint32_t ph = (h | (h >> 4)) & 0x00FF00FFu;
+    return (pl & 0xFFu) | ((pl >> 8) & 0xFF00u) | ((ph & 0xFFu) << 16) | ((ph >> 8) & 0xFF00u) << 16;
+  };
+  const uint4 out = make_uint4(pack8(a.x, a.y), pack8(a.z, a.w), pack8(b.x, b.y), pack8(b.z, b.w));
+  *reinterpret_cast<uint4*>(packed + i * 16) = out;
+}
+
+int launch_pack_codes4(const uint8_t* codes, int64_t n_codes, uint8_t* packed, cudaStream_t st) {
+  const int64_t packets = n_codes / 32;
+  pack_codes4_kernel<<<(unsigned)ceil_div(packets, 256), 256, 0, st>>>(codes, packets, packed);
+  return after_launch();
+}
+
 }  // namespace tlq

@@ -29,7 +29,7 @@ STAGE_NAMES = ("stats", "fakequant", "gemm", "reduce")
 
 EXPORTS = (
     "tlq_status_string", "tlq_version", "tlq_token_importance", "tlq_scale_candidates_workspace_bytes",
-    "tlq_scale_candidates", "tlq_scale_candidates_noalloc", "tlq_quantize_weights", "tlq_quantize_activations", "tlq_scale_search_workspace_bytes", "tlq_scale_search_layer", "tlq_scale_search_layer_two_stream",
+    "tlq_scale_candidates", "tlq_scale_candidates_noalloc", "tlq_quantize_weights", "tlq_pack_codes4", "tlq_quantize_activations", "tlq_scale_search_workspace_bytes", "tlq_scale_search_layer", "tlq_scale_search_layer_two_stream",
     "tlq_apply_layer_workspace_bytes", "tlq_apply_layer", "tlq_read_status", "tlq_stage_timing_enable",
     "tlq_stage_timing_drain", "tlq_kernel_launch_count",
 )
@@ -79,6 +79,8 @@ def _load() -> ctypes.CDLL:
     lib.tlq_scale_candidates_noalloc.argtypes = [vp, i64, i64, vp, cfgp, vp, vp, vp]
     lib.tlq_scale_candidates_noalloc.restype = i32
     lib.tlq_quantize_weights.argtypes = [vp, vp, i64, i64, cfgp, vp, vp, vp, vp, vp]
+    lib.tlq_pack_codes4.argtypes = [vp, i64, i64, vp, vp]
+    lib.tlq_pack_codes4.restype = i32
     lib.tlq_quantize_activations.argtypes = [vp, vp, i64, i64, cfgp, vp, vp, vp]
     lib.tlq_quantize_activations.restype = i32
     lib.tlq_scale_search_workspace_bytes.restype = sz
@@ -92,7 +94,7 @@ def _load() -> ctypes.CDLL:
     lib.tlq_read_status.argtypes = [vp, vp]
     lib.tlq_stage_timing_enable.argtypes = [i32]
     lib.tlq_stage_timing_drain.argtypes = [ctypes.POINTER(ctypes.c_float), i32]
-    for fn in ("tlq_token_importance", "tlq_scale_candidates", "tlq_scale_candidates_noalloc", "tlq_quantize_weights", "tlq_quantize_activations", "tlq_scale_search_layer",
+    for fn in ("tlq_token_importance", "tlq_scale_candidates", "tlq_scale_candidates_noalloc", "tlq_quantize_weights", "tlq_pack_codes4", "tlq_quantize_activations", "tlq_scale_search_layer",
                "tlq_apply_layer", "tlq_read_status", "tlq_stage_timing_enable", "tlq_stage_timing_drain"):
         getattr(lib, fn).restype = i32
     return lib
@@ -178,6 +180,14 @@ def tlq_quantize_weights(W: torch.Tensor, s: Optional[torch.Tensor], cfg: Config
     _check(lib.tlq_quantize_weights(_ptr(W), _ptr(s), C2, C1, ctypes.byref(cfg), _ptr(codes), _ptr(steps), _ptr(zeros),
                                     _ptr(dW), _stream(stream)), "tlq_quantize_weights")
     return dict(codes=codes, steps=steps, zeros=zeros, dW=dW)
+
+
+def tlq_pack_codes4(codes: torch.Tensor, stream=None) -> torch.Tensor:
+    """codes uint8/int8 [R,C] (one 4-bit code per byte) -> uint8 [R,C/2], even channel in the low nibble."""
+    R, C = codes.shape
+    packed = torch.empty((R, C // 2), dtype=torch.uint8, device=codes.device)
+    _check(lib.tlq_pack_codes4(_ptr(codes), R, C, _ptr(packed), _stream(stream)), "tlq_pack_codes4")
+    return packed
 
 
 def tlq_quantize_activations(X: torch.Tensor, s: Optional[torch.Tensor], cfg: Config, stream=None):

@@ -565,3 +565,17 @@ def test_grid_of_one_and_of_the_maximum(tlq, mode, n_grid):
     if n_grid == 1:
         assert got["best"] == 0 and np.all(wl.bf16_bits_to_f32(got["s_best"]) == 1.0)
     assert tlq.tlq_scale_search_workspace_bytes(200, 128, 96, tlq.config(n_grid=65)) == 0
+
+
+def test_four_bit_packing_bit_exact(tlq):
+    wb = wl.weights(161, "pack/w", 77, 1056)
+    s_np = orc.scale_table(orc.channel_stat(wl.activations(161, "pack/x", 64, 1056, 48)), 20)[7]
+    s_dev = dev_bf16(tlq, orc.f32_to_bf16_bits(s_np))
+    out = tlq.tlq_quantize_weights(dev_bf16(tlq, wb), s_dev, tlq.config(group_size=32))
+    codes, _, _, _ = orc.quantize_weights_group_asym(wb, s_np, 32, 4)
+    assert np.array_equal(tlq.tlq_pack_codes4(out["codes"]).cpu().numpy(), orc.pack_codes4(codes))
+    sym = tlq.tlq_quantize_weights(dev_bf16(tlq, wb), s_dev, tlq.config(tlq.WA_SYM_CHANNEL, w_bits=4, a_bits=8))
+    qw, _ = orc.quantize_weights_row_sym(wb, s_np, 4)
+    packed = tlq.tlq_pack_codes4(sym["codes"]).cpu().numpy()
+    assert np.array_equal(packed, orc.pack_codes4(qw))
+    assert np.array_equal(orc.unpack_codes4(packed, signed=True), qw)

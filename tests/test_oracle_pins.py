@@ -439,3 +439,15 @@ def test_two_stream_objective(mode):
             _, _, _, w_hat = orc.quantize_weights_group_asym(w, two["scales"][k], 4)
             e = d + orc.bf16_to_f64(xq) @ (orc.bf16_to_f64(w) - w_hat.astype(np.float64)).T
             assert np.allclose(two["per_token"][k], (e ** 2).sum(axis=1), rtol=1e-9)
+
+
+def test_four_bit_packing_round_trips():
+    x, w, _ = wl.small_case(151, 8, 64, 6)
+    s = orc.scale_table(orc.channel_stat(x), 20)[9]
+    codes, _, _, _ = orc.quantize_weights_group_asym(w, s, 32, 4)
+    packed = orc.pack_codes4(codes)
+    assert packed.shape == (6, 32) and packed.dtype == np.uint8
+    assert np.array_equal(orc.unpack_codes4(packed, signed=False), codes)
+    assert packed[0, 0] == (int(codes[0, 0]) | (int(codes[0, 1]) << 4))          # even channel in the low nibble
+    qw, _ = orc.quantize_weights_row_sym(w, s, 4)
+    assert np.array_equal(orc.unpack_codes4(orc.pack_codes4(qw), signed=True), qw)
