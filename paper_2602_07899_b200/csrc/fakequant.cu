@@ -156,13 +156,14 @@ fakequant_delta_kernel(const uint16_t* __restrict__ W, const uint16_t* __restric
   uint4 (*tile)[kGqCols / 8] = reinterpret_cast<uint4 (*)[kGqCols / 8]>(tile_dyn);
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
-  const int64_t c0 = (int64_t)blockIdx.x * kGqCols + lane * 16;
-  const int64_t row0 = (int64_t)blockIdx.y * kHotRows;
+  const int64_t col_blocks = (C1 + kGqCols - 1) / kGqCols;      // grid.x = column blocks x row tiles, columns fastest
+  const int64_t c0 = (int64_t)(blockIdx.x % col_blocks) * kGqCols + lane * 16;
+  const int64_t row0 = (int64_t)(blockIdx.x / col_blocks) * kHotRows;
   const bool col_ok = c0 < C1;
   const int lanes_per_group = group >> 4;
   const float qmax_f = (float)qmax;
   const float tie_lim = 0.5f - tie_eps;
-  const int k_begin = blockIdx.z * k_per_cta;
+  const int k_begin = blockIdx.y * k_per_cta;
   const int k_end = min(K, k_begin + k_per_cta);
 
 #pragma unroll
@@ -285,13 +286,14 @@ fakequant_group_kernel(const uint16_t* __restrict__ W, const uint16_t* __restric
   __shared__ uint4 tile[kGqRows][kGqCols / 8];
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
-  const int64_t c0 = (int64_t)blockIdx.x * kGqCols + lane * 16;
-  const int64_t row0 = (int64_t)blockIdx.y * kGqRows;
+  const int64_t col_blocks = (C1 + kGqCols - 1) / kGqCols;      // grid.x = column blocks x row tiles, columns fastest
+  const int64_t c0 = (int64_t)(blockIdx.x % col_blocks) * kGqCols + lane * 16;
+  const int64_t row0 = (int64_t)(blockIdx.x / col_blocks) * kGqRows;
   const bool col_ok = c0 < C1;                    // C1 % 16 == 0 is guaranteed by the group sizes
   const int lanes_per_group = group >> 4;
   const float qmax_f = (float)qmax;
   const int64_t ngroups = C1 / group;
-  const int k_begin = blockIdx.z * k_per_cta;
+  const int k_begin = blockIdx.y * k_per_cta;
   const int k_end = min(K, k_begin + k_per_cta);
 
   // stage the W tile (zeros outside the matrix)
@@ -407,7 +409,7 @@ int launch_fakequant_group(const uint16_t* W, const uint16_t* s, const float* rs
   if (kchunks < 1) kchunks = 1;
   const int k_per_cta = (int)ceil_div(K, kchunks);
   kchunks = ceil_div(K, k_per_cta);
-  dim3 grid((unsigned)ceil_div(C1, kGqCols), (unsigned)ceil_div(C2, tile_rows), (unsigned)kchunks);
+  dim3 grid((unsigned)(ceil_div(C1, kGqCols) * ceil_div(C2, tile_rows)), (unsigned)kchunks);
   if (hot) {
     static bool configured = false;
     if (!configured) {
@@ -505,13 +507,14 @@ row_amax_kernel(const uint16_t* __restrict__ src, const uint16_t* __restrict__ s
   extern __shared__ uint4 tile_dyn[];
   uint4 (*tile)[kGqCols / 8] = reinterpret_cast<uint4 (*)[kGqCols / 8]>(tile_dyn);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int64_t c0 = (int64_t)blockIdx.x * kGqCols + lane * 16;
-  const int64_t row0 = (int64_t)blockIdx.y * kRowRows;
+  const int64_t col_blocks = (C1 + kGqCols - 1) / kGqCols;      // grid.x = column blocks x row tiles, columns fastest
+  const int64_t c0 = (int64_t)(blockIdx.x % col_blocks) * kGqCols + lane * 16;
+  const int64_t row0 = (int64_t)(blockIdx.x / col_blocks) * kRowRows;
   const int64_t R = (n_rows_dev != nullptr) ? (int64_t)*n_rows_dev : R_all;    // rows beyond are not live
   if (row0 >= R) return;                                                        // the whole CTA leaves together
   const bool col_ok = c0 < C1;
   stage_tile(tile, src, row0, R, C1, c0, col_ok, warp, lane);
-  const int k_begin = blockIdx.z * k_per_cta;
+  const int k_begin = blockIdx.y * k_per_cta;
   const int k_end = min(K, k_begin + k_per_cta);
   for (int k = k_begin; k < k_end; ++k) {
     float2 m[8];
@@ -579,8 +582,9 @@ row_codes_kernel(const uint16_t* __restrict__ src, const uint16_t* __restrict__ 
   extern __shared__ uint4 tile_dyn[];
   uint4 (*tile)[kGqCols / 8] = reinterpret_cast<uint4 (*)[kGqCols / 8]>(tile_dyn);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int64_t c0 = (int64_t)blockIdx.x * kGqCols + lane * 16;
-  const int64_t row0 = (int64_t)blockIdx.y * kRowRows;
+  const int64_t col_blocks = (C1 + kGqCols - 1) / kGqCols;      // grid.x = column blocks x row tiles, columns fastest
+  const int64_t c0 = (int64_t)(blockIdx.x % col_blocks) * kGqCols + lane * 16;
+  const int64_t row0 = (int64_t)(blockIdx.x / col_blocks) * kRowRows;
   const int64_t R = (n_rows_dev != nullptr) ? (int64_t)*n_rows_dev : R_all;
   if (row0 >= R) return;
   const bool col_ok = c0 < C1;
@@ -588,7 +592,7 @@ row_codes_kernel(const uint16_t* __restrict__ src, const uint16_t* __restrict__ 
   if (!col_ok) return;                    // no warp-wide operation below
   const float tie_lim = 0.5f - tie_eps;
   const float2 magic2 = make_float2(kMagic, kMagic);
-  const int k_begin = blockIdx.z * k_per_cta;
+  const int k_begin = blockIdx.y * k_per_cta;
   const int k_end = min(K, k_begin + k_per_cta);
   for (int k = k_begin; k < k_end; ++k) {
     float2 m[8];
@@ -648,7 +652,7 @@ static int launch_rows(const uint16_t* src, const uint16_t* s, const float* rs, 
   if (kchunks < 1) kchunks = 1;
   const int k_per_cta = (int)ceil_div(K, kchunks);
   kchunks = ceil_div(K, k_per_cta);
-  const dim3 grid((unsigned)ceil_div(C1, kGqCols), (unsigned)ceil_div(R, kRowRows), (unsigned)kchunks);
+  const dim3 grid((unsigned)(ceil_div(C1, kGqCols) * ceil_div(R, kRowRows)), (unsigned)kchunks);
   const float qpos = (float)((1 << (bits - 1)) - 1);
   const float tie_eps = 4.0e-7f * (qpos + 1.0f);
   const int64_t n = (int64_t)K * R;
