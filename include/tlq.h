@@ -13,7 +13,8 @@
  *  - Every pointer is a DEVICE pointer unless its comment says "host".  The caller owns all buffers;
  *    the library allocates and frees no device memory.  bf16 tensors are raw uint16 bit patterns,
  *    row-major, innermost dimension contiguous.  X, W and the workspace must be 16-byte aligned
- *    (TMA base-address rule) and C1 must be a multiple of 8 (16-byte row pitch).
+ *    (TMA base-address rule) and C1 must be a multiple of 8 (16-byte row pitch), of 16 in the
+ *    symmetric mode (16-byte rows of int8 codes) and of the group size in the group mode.
  *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls validate
  *    their arguments on the host, enqueue kernels on `stream` and return without synchronising.
  *  - Return value: TLQ_OK or a negative TLQ_ERR_* for errors found on the host.  Errors found on

@@ -162,7 +162,7 @@ const char* tlq_status_string(int status) {
   }
 }
 
-int tlq_version(void) { return 1000; }
+int tlq_version(void) { return 1004; }   // 1.4: symmetric widths, flags, two-stream search, 4-bit packing
 
 int64_t tlq_kernel_launch_count(void) { return (int64_t)g_launch_count; }
 
