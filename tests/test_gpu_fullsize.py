@@ -155,3 +155,42 @@ def test_2b_64k_tokens_sampled(tlq, mode):
     assert np.array_equal(got["s_best"], orc.f32_to_bf16_bits(scales[got["best"]]))
     tokens = np.sort(np.random.default_rng(3).choice(cfgw.n_tokens, 96, replace=False))
     check_sampled(got, cfgw, xb, wb, scales, tokens, (0, 8, 19))
+
+
+def test_7b_k_projection_full_paper_settings(tlq):
+    """The paper's own setting on the 7B k-projection at full size: W4A8 with the top-50 % token set as 0/1
+    weights, zero-weight tokens skipped on the device."""
+    cfgw = wl.config("cfg1", mode="w4a8")
+    data = wl.LayerData(cfgw)
+    lin = cfgw.linear("k")
+    xb, wb, imp = data.x(lin), data.w(lin), data.imp()
+    mask = (imp >= np.sort(imp)[len(imp) // 2]).astype(np.float32)
+    ref = orc.scale_search(xb, wb, mask, "w4a8", 0, cfgw.n_grid)
+    cfg = tlq.config(tlq.WA_SYM_CHANNEL, w_bits=4, a_bits=8, n_grid=cfgw.n_grid, flags=tlq.FLAG_SKIP_ZERO_WEIGHT_TOKENS)
+    out = tlq.tlq_scale_search_layer(tlq.bf16_from_bits(xb), tlq.bf16_from_bits(wb), torch.from_numpy(mask).cuda(), cfg)
+    np.testing.assert_allclose(out.losses.cpu().numpy(), ref["losses"], rtol=LOSS_RTOL)
+    order = np.sort(ref["losses"])
+    if (order[1] - order[0]) / order[0] > 1e-5:
+        assert int(out.best_idx.item()) == ref["best"]
+
+
+@pytest.mark.parametrize("key", ["cfg1", "cfg2"])
+def test_7b_k_projection_full_two_streams(tlq, key):
+    """Two activation streams at full size: the quantized stream is the full-precision one with a 2 % relative
+    perturbation (rounded to bf16)."""
+    cfgw = wl.config(key)
+    data = wl.LayerData(cfgw)
+    lin = cfgw.linear("k")
+    xf, wb, imp = data.x(lin), data.w(lin), data.imp()
+    noise = np.random.default_rng(9).standard_normal(xf.shape).astype(np.float32)
+    xq = wl.f32_to_bf16_bits(wl.bf16_bits_to_f32(xf) * (1.0 + 0.02 * noise))
+    ref = orc.scale_search(xq, wb, imp, cfgw.mode, cfgw.group, cfgw.n_grid, x_fp_bits=xf)
+    mode = tlq.W4A16_ASYM_GROUP if cfgw.mode == "w4a16" else tlq.W8A8_SYM
+    cfg = tlq.config(mode=mode, group_size=cfgw.group, n_grid=cfgw.n_grid)
+    out = tlq.tlq_scale_search_layer(tlq.bf16_from_bits(xq), tlq.bf16_from_bits(wb), torch.from_numpy(imp).cuda(), cfg,
+                                     per_token=True, X_fp=tlq.bf16_from_bits(xf))
+    np.testing.assert_allclose(out.per_token.cpu().numpy(), ref["per_token"], rtol=LOSS_RTOL, atol=1e-30)
+    np.testing.assert_allclose(out.losses.cpu().numpy(), ref["losses"], rtol=LOSS_RTOL)
+    order = np.sort(ref["losses"])
+    if (order[1] - order[0]) / order[0] > 1e-5:
+        assert int(out.best_idx.item()) == ref["best"]
