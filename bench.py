@@ -221,6 +221,25 @@ def run_ours(args, cfgw):
     cfgr = dataclasses.replace(cfgw, seed=replicas.replica_seed(cfgw.seed, rank))
     data = wl.LayerData(cfgr)
     lins = [l for l in cfgr.linears() if args.linears is None or l.name in args.linears.split(",")]
+    n_linears = len(lins)
+    stacked = {}
+    if args.shared_scale:
+        # linears fed by the same activations share one scale (it is folded into the layer before them): their
+        # weight matrices are stacked row-wise and searched as one; the step still covers all seven linears
+        groups = {}
+        for l in lins:
+            groups.setdefault(l.x_name, []).append(l)
+        lins = []
+        for x_name, members in groups.items():
+            name = "+".join(m.name for m in members)
+            lins.append(wl.Linear(name, members[0].c_in, sum(m.c_out for m in members), x_name))
+            stacked[name] = members
+
+    def weights_of(l):
+        if l.name in stacked:
+            return np.concatenate([data.w(m) for m in stacked[l.name]], axis=0)
+        return data.w(l)
+
     flags = tlq.FLAG_SKIP_ZERO_WEIGHT_TOKENS if args.skip_zero_weight else 0
     flags |= {"default": 0, "pairs": tlq.FLAG_GEMM_CTA_PAIRS, "narrow": tlq.FLAG_GEMM_NARROW_TILES}[args.gemm]
     if cfgr.mode == "w4a16":
@@ -235,7 +254,7 @@ def run_ours(args, cfgw):
         if l.x_name not in host_x:
             host_x[l.x_name] = torch.from_numpy(data.x(l).view(np.int16)).pin_memory()
             dev_x[l.x_name] = host_x[l.x_name].to(dev, non_blocking=True).view(torch.bfloat16)
-        host_w[l.name] = torch.from_numpy(data.w(l).view(np.int16)).pin_memory()
+        host_w[l.name] = torch.from_numpy(weights_of(l).view(np.int16)).pin_memory()
         dev_w[l.name] = host_w[l.name].to(dev, non_blocking=True).view(torch.bfloat16)
     imp_np = data.imp()
     if args.importance == "top50":      # the paper's token set: 1 for the top half by importance, 0 for the rest
@@ -317,7 +336,7 @@ def run_ours(args, cfgw):
     # ---- max over ranks
     ms_total, ms_e2e = replicas.max_over_ranks([ms_total, ms_e2e], info, dev)
 
-    n_cand_step = len(lins) * cfgr.n_grid
+    n_cand_step = n_linears * cfgr.n_grid
     value = replicas.whole_job_rate(n_cand_step, args.steps, info, ms_total)
     e2e_value = replicas.whole_job_rate(n_cand_step, args.steps, info, ms_e2e)
 
@@ -360,7 +379,7 @@ def run_ours(args, cfgw):
     traffic = None
     tpath = os.path.join(ROOT, "profiles", "search_gemm_traffic.json")
     if os.path.exists(tpath) and args.linears is None and args.mode is None and not args.skip_zero_weight \
-            and args.gemm == "default":
+            and args.gemm == "default" and not args.shared_scale:
         with open(tpath) as f:      # ncu counters of this very workload and kernel; anything else has none
             traffic = json.load(f).get(cfgr.key)
     i8 = cfgr.mode != "w4a16"
@@ -393,7 +412,7 @@ def run_ours(args, cfgw):
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if cfgr.mode == "w4a16" else "int8", "data": "synthetic",
-            "config": {"workload": workload_name(cfgr) + ("" if args.linears is None else f" [subset: {args.linears}]") + ("" if args.importance == "config" else f" [importance: {args.importance}]") + (" [zero-weight tokens skipped]" if args.skip_zero_weight else ""), "l2": "inputs_exceed_l2 (operands of one linear: 0.1-2.9 GB)",
+            "config": {"workload": workload_name(cfgr) + ("" if args.linears is None else f" [subset: {args.linears}]") + ("" if args.importance == "config" else f" [importance: {args.importance}]") + (" [zero-weight tokens skipped]" if args.skip_zero_weight else "") + (" [shared scale: " + ", ".join(l.name for l in lins) + "]" if args.shared_scale else ""), "l2": "inputs_exceed_l2 (operands of one linear: 0.1-2.9 GB)",
                        "parallelism": f"replicas x{world} (one layer per rank, no collective)"},
             "gemm_tflops": achieved, "roofline": roofline, "cpu_baseline": cpu,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -418,6 +437,8 @@ def main():
                     help="set TLQ_FLAG_SKIP_ZERO_WEIGHT_TOKENS (tensor FLOP/s then count the live tokens only)")
     ap.add_argument("--gemm", default="default", choices=["default", "pairs", "narrow"],
                     help="variant of the bf16 search GEMM (TLQ_FLAG_GEMM_*), for A/B measurements")
+    ap.add_argument("--shared-scale", action="store_true",
+                    help="stack linears that share their input (q/k/v, gate/up) and search one scale for each stack")
     ap.add_argument("--linears", default=None, help="comma-separated subset of q,k,v,o,gate,up,down (profiling)")
     ap.add_argument("--profile", action="store_true", help="kernel leg only: skip the end-to-end and CPU legs")
     args = ap.parse_args()
