@@ -66,6 +66,39 @@ __device__ __forceinline__ void report_timeout(WorkspaceHeader* hdr, int where) 
   hdr->status = TLQ_ERR_TIMEOUT;
 }
 
+// What one CTA does next.  Whole waves of tiles run all K candidates per tile; the tiles left over for the last,
+// partial wave are split by candidates over the CTAs that would otherwise idle (each split recomputes the
+// candidate-free tile, two pass-equivalents, against up to K passes saved): with 896 tiles on 148 SMs the seventh
+// wave of 8 tiles costs 3 pass-times instead of 22.
+struct TailSplit {
+  int full;        // tiles handled whole (a multiple of the grid size)
+  int chunks;      // candidate chunks per left-over tile
+  int per;         // candidates per chunk
+  int items;       // left-over tiles x chunks (<= grid size)
+};
+__device__ __forceinline__ TailSplit make_tail_split(int num_tiles, int grid, int K) {
+  TailSplit t;
+  t.full = (num_tiles / grid) * grid;
+  const int rest = num_tiles - t.full;
+  int splits = rest > 0 ? grid / rest : 1;
+  if (splits > K) splits = K;
+  if (splits < 1) splits = 1;
+  t.per = (K + splits - 1) / splits;
+  t.chunks = (K + t.per - 1) / t.per;
+  t.items = rest * t.chunks;
+  return t;
+}
+// Work item number w of this launch -> (tile, candidates [k0, k1)); false when there is none.
+__device__ __forceinline__ bool work_item(const TailSplit& t, int w, int K, int& tile, int& k0, int& k1) {
+  if (w < t.full) { tile = w; k0 = 0; k1 = K; return true; }
+  const int j = w - t.full;
+  if (j >= t.items) return false;
+  tile = t.full + j / t.chunks;
+  k0 = (j % t.chunks) * t.per;
+  k1 = k0 + t.per < K ? k0 + t.per : K;
+  return true;
+}
+
 // kMode 0: W8A8-style search (one bf16 pass for the full-precision tile, then K int8 passes)
 // kMode 1: apply (a single int8 pass, bf16 store)
 // kMode 2: two-stream search with 16-bit activations (first propagation strategy of paper Sec. 3.2.1):
@@ -116,7 +149,7 @@ gemm_w8a8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
   const uint32_t tmem_base = *tmem_slot;
 
   // pass 0 of a search tile is the full-precision product; apply has the single int8 pass only
-  const int passes = kApply ? 1 : args.K + 1;
+  const int n_cand = kApply ? 1 : args.K;      // passes of one work item: its candidates (+ the candidate-free pass)
   // token count and tile walk: fixed by the host, or read from the device when the tokens were compacted
   int64_t n_tokens = args.N, num_tiles = args.num_tiles;
   TileRaster raster = args.raster;
@@ -128,18 +161,23 @@ gemm_w8a8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     num_tiles = args.otiles * mt_live;
   }
 
+  const TailSplit split = make_tail_split((int)num_tiles, (int)gridDim.x, n_cand);
+
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+      for (int w = blockIdx.x; ok; w += gridDim.x) {
+        int tile, k0, k1;
+        if (!work_item(split, w, n_cand, tile, k0, k1)) break;
+        const int passes = kApply ? 1 : k1 - k0 + 1;
         int mt, ot;
         raster.decode(tile, mt, ot);
         for (int pass = 0; pass < passes && ok; ++pass) {
           const bool fp = !kApply && pass == 0;
-          const int k = kApply ? 0 : pass - 1;
+          const int k = kApply ? 0 : k0 + pass - 1;
           const int nkb = fp ? (kDual ? 2 * args.num_kb16 : args.num_kb16) : (kDual ? args.num_kb16 : args.num_kb8);
           for (int kb = 0; kb < nkb; ++kb) {
             if (!ptx::mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
@@ -175,7 +213,10 @@ gemm_w8a8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       uint32_t phase = 0;
       int64_t it = 0;                      // passes issued so far: selects the accumulator
       bool ok = true;
-      for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+      for (int w = blockIdx.x; ok; w += gridDim.x) {
+        int tile, k0, k1;
+        if (!work_item(split, w, n_cand, tile, k0, k1)) break;
+        const int passes = kApply ? 1 : k1 - k0 + 1;
         for (int pass = 0; pass < passes && ok; ++pass, ++it) {
           const bool fp = !kApply && pass == 0;
           const int nkb = fp ? (kDual ? 2 * args.num_kb16 : args.num_kb16) : (kDual ? args.num_kb16 : args.num_kb8);
@@ -224,7 +265,10 @@ gemm_w8a8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     float yfp[128];                               // this thread's share of the full-precision tile
     int64_t it = 0;
     bool ok = true;
-    for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+    for (int w = blockIdx.x; ok; w += gridDim.x) {
+      int tile, k0, k1;
+      if (!work_item(split, w, n_cand, tile, k0, k1)) break;
+      const int passes = kApply ? 1 : k1 - k0 + 1;
       int mt, ot;
       raster.decode(tile, mt, ot);
       const int64_t n = (int64_t)mt * BM + row_in_tile;
@@ -253,7 +297,7 @@ gemm_w8a8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
           if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
           continue;
         }
-        const int k = kApply ? 0 : pass - 1;
+        const int k = kApply ? 0 : k0 + pass - 1;
         const float tn = (!kDual && n < n_tokens) ? args.t[(int64_t)k * args.N + n] : 0.0f;
         const float* u_row = kDual ? nullptr : args.u + (int64_t)k * args.C2;
         if (!kApply) {
