@@ -3,6 +3,8 @@
 #include <math.h>
 #include <string.h>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "common.cuh"
 
 namespace tlq {
@@ -123,7 +125,13 @@ int g_ev_made = 0;      // sets whose events exist
 int g_calls = 0;        // calls recorded since the last enable
 int g_cur = -1;         // set being recorded by the call in progress
 
+// Stage boundaries of a search call: a named range for timeline profilers (host side: the range covers the
+// enqueueing of the stage; free when no tool is attached) and, when stage timing is on, an event on the stream.
+const char* const kStageNames[TLQ_N_STAGES] = {"tlq.stats", "tlq.fakequant", "tlq.gemm", "tlq.reduce"};
+
 int timing_mark(int i, cudaStream_t st) {
+  if (i > 0) nvtxRangePop();
+  if (i < TLQ_N_STAGES) nvtxRangePushA(kStageNames[i]);
   if (!g_timing_on) return TLQ_OK;
   if (i == 0) {
     if (g_calls >= kMaxTimedCalls) { g_cur = -1; return TLQ_OK; }
