@@ -358,6 +358,7 @@ def run_ours(args, cfgw):
         gemm_flops_sum += fl
     n_rec = max(1, len(stage_ms) // len(lins))
     lin_report = {}
+    stream_tot = {"stats": [0.0, 0.0], "fakequant": [0.0, 0.0]}     # algorithmic bytes, ms per step
     for name, d in per_linear.items():
         g = statistics.mean(d["gemm_ms"])
         l = next(x for x in lins if x.name == name)
@@ -369,6 +370,10 @@ def run_ours(args, cfgw):
             fq_bytes = (2.0 + 2.0 * K) * l.c_out * l.c_in
         else:
             fq_bytes = (2.0 + K) * l.c_out * l.c_in + (2.0 + K) * cfgr.n_tokens * l.c_in
+        stream_tot["stats"][0] += stat_bytes
+        stream_tot["stats"][1] += d["stages_ms"][0] / n_rec
+        stream_tot["fakequant"][0] += fq_bytes
+        stream_tot["fakequant"][1] += d["stages_ms"][1] / n_rec
         lin_report[name] = {"gemm_ms": round(g, 4), "gemm_tflops": round(d["flops"] / (g * 1e-3) / 1e12, 1),
                             "stats_gbs": round(stat_bytes / (d["stages_ms"][0] / n_rec * 1e-3) / 1e9, 1),
                             "fakequant_gbs": round(fq_bytes / (d["stages_ms"][1] / n_rec * 1e-3) / 1e9, 1),
@@ -417,7 +422,13 @@ def run_ours(args, cfgw):
             "gemm_tflops": achieved, "roofline": roofline, "cpu_baseline": cpu,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": ms_e2e / args.steps},
-            "gpu_launches": launches, "clocks": clocks, "per_linear": lin_report, "other_path_steps": extra}
+            "gpu_launches": launches, "clocks": clocks, "per_linear": lin_report, "other_path_steps": extra,
+            "streaming_stages": {n: {"bound": "hbm", "achieved": round(b / (ms * 1e-3) / 1e9, 1) if ms > 0 else None,
+                                     "peak": peaks["hbm"], "unit": "GB/s",
+                                     "frac": round(b / (ms * 1e-3) / 1e9 / peaks["hbm"], 3) if ms > 0 else None,
+                                     "note": "algorithmic bytes of the stage over its in-step time (events between "
+                                             "stages: includes launch gaps; the kernels are issue-bound, not HBM-bound)"}
+                                 for n, (b, ms) in stream_tot.items()}}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
