@@ -9,7 +9,7 @@ What the paper fixes, and where each function comes from:
   * quantizer: X_hat = round(X / s_i), s_i = max_j |X_ij| / (2^(n-1) - 1), integers in
     [-2^(n-1), 2^(n-1)-1]; per token for activations, per output channel for weights
     (Sec. 2.2, first two equations and the integer-range sentence).  The asymmetric variant
-    "follows in a similar manner" (same section); its formula here is a reading (min/max affine grid).
+    is only said to be handled analogously (same section); its formula here is a reading (min/max affine grid).
   * smoothing: Y = (X diag(scale)^-1)(diag(scale) W) (Sec. 2.2, per-channel smoothing equation);
     scale indexes the input channels of W in R^{C2 x C1}.
   * scale = x_stat^r (Sec. 3.1.2, first equation), x_stat_c = max over the selected tokens of
