@@ -16,8 +16,9 @@ What the paper fixes, and where each function comes from:
     |X_ic| (second equation), with mean / max over all tokens as the ablation variants (Table 2).
   * search: r* = argmin_r E || f_fp(x) - f_q(x; scale) ||^2, f_fp = W x + b,
     f_q = Q_w(W * scale) Q_a(x / scale) + b (Sec. 3.2.1).
-  * token importance: sum_n = sum_b ||g_{b,n}|| with the text's "absolute values, mean over the
-    channel dimension"; I = Top50% (Sec. 3.1.2, last two equations).
+  * token importance: sum_n = sum_b ||g_{b,n}||, where the surrounding text describes the norm as the
+    channel mean of the absolute gradient; I = the top half of the tokens by sum_n (Sec. 3.1.2, last two
+    equations).
 
 Contract points (where floating point decides an integer the decision is taken in binary32, the
 precision of the CUDA kernels; everything else is float64): the product scale*w (exact in binary32
