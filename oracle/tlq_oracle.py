@@ -26,12 +26,15 @@ for bf16 factors), the group range, the step, the zero-point quotient, the code 
 dequantized value, the reciprocal of the scale and the product with it.  They are written with
 numpy float32 arrays, one IEEE operation per statement.
 
-Readings of silent points (the grid r_k = k/K, bf16 storage of the scale, half-to-even rounding,
-floors on degenerate statistics, loss normalisation by C2 * sum(w)) are listed in the design notes.
+Readings of points the paper leaves open, each stated where it is used below: the grid r_k = k/K
+(grid_ratio), bfloat16 storage of the scale (scale_table), half-to-even rounding (np.rint), the floors
+on degenerate statistics (_STAT_FLOOR, _RANGE_FLOOR), diag(scale)^-1 taken as a product with the
+binary32 reciprocal (quantize_weights_group_asym, quantize_activations_token_sym) and the loss
+normalisation by C2 * sum(w) (weighted_loss).
 
-Parity pins: see tests/test_oracle_pins.py (closed forms, invariants, brute force on tiny inputs).
-The paper prints no worked numeric example for any function here, so absolute values are pinned
-only by those tests.
+Parity pins: tests/test_oracle_pins.py holds, for every function here, closed forms, hand-computed
+values, invariants, library conversions or a scalar brute force on tiny inputs.  The paper prints no
+worked numeric example, so absolute values are pinned by those tests alone.
 """
 from __future__ import annotations
 

@@ -451,3 +451,152 @@ def test_four_bit_packing_round_trips():
     assert packed[0, 0] == (int(codes[0, 0]) | (int(codes[0, 1]) << 4))          # even channel in the low nibble
     qw, _ = orc.quantize_weights_row_sym(w, s, 4)
     assert np.array_equal(orc.unpack_codes4(orc.pack_codes4(qw), signed=True), qw)
+
+
+# ------------------------------------------------------------------ delta-weight operand, symmetric apply, reciprocal reading
+
+
+def test_delta_weights_bf16_hand_values():
+    """W - W_hat, one rounding to binary32 and one to bfloat16 (ties to even), checked on values worked out by hand:
+    operand order and sign, a value already representable, both kinds of bfloat16 tie, and a case where the
+    binary32 rounding lands on a tie that a single rounding from the exact difference would not see."""
+    def one(w, w_hat):
+        return int(orc.delta_weights_bf16(bits([[w]]), np.array([[w_hat]], dtype=np.float32))[0, 0])
+    assert one(1.0, 0.75) == 0x3E80                       # +0.25
+    assert one(0.5, 0.75) == 0xBE80                       # -0.25: W minus W_hat, not the reverse
+    assert one(-1.0, -0.75) == 0xBE80
+    assert one(0.25, 0.25) == 0x0000                      # no error -> +0
+    # 2^-4 (1 + 2^-8): halfway between mantissas 0 and 1 -> even mantissa 0
+    assert one(1.0, 1.0 - 2.0 ** -4 - 2.0 ** -12) == 0x3D80
+    # 2^-4 (1 + 3 * 2^-8): halfway between mantissas 1 and 2 -> even mantissa 2
+    assert one(1.0, 1.0 - 2.0 ** -4 - 3 * 2.0 ** -12) == 0x3D82
+    # just above / below the first tie
+    assert one(1.0, 1.0 - 2.0 ** -4 - 2.0 ** -12 - 2.0 ** -20) == 0x3D81
+    assert one(1.0, 1.0 - 2.0 ** -4 - 2.0 ** -12 + 2.0 ** -20) == 0x3D80
+    # exact difference 1 + 2^-8 + 2^-26: binary32 drops the 2^-26 (below half an ulp of 2^-23), leaving the tie
+    # 1 + 2^-8, which goes to the even mantissa 0; one rounding from the exact value would give 1 + 2^-7
+    w_hat = np.float32(2.0 ** -8 - 2.0 ** -26)
+    assert float(w_hat) == 2.0 ** -8 - 2.0 ** -26
+    assert one(1.0 + 2.0 ** -7, float(w_hat)) == 0x3F80
+    # the same through a library conversion chain on random data (float32 subtraction, then torch's bf16 rounding)
+    rng = np.random.default_rng(12)
+    wb = bits(rng.standard_normal((16, 64)) * 0.02)
+    w_hat = (wl.bf16_bits_to_f32(wb) + rng.standard_normal((16, 64)).astype(np.float32) * np.float32(1e-3)).astype(np.float32)
+    ref = torch.from_numpy(wl.bf16_bits_to_f32(wb) - w_hat).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(orc.delta_weights_bf16(wb, w_hat), ref)
+
+
+def test_delta_weights_reproduce_the_candidate_error():
+    """The bf16 delta-weight operand is a rounding of W - W_hat: X dW^T reproduces the search's per-token error to
+    the operand's rounding (half an ulp of an 8-bit significand: 2^-8 relative) (a sign or transposition slip would be off by orders of magnitude)."""
+    x, w, imp = wl.small_case(181, 48, 128, 24)
+    res = orc.scale_search(x, w, imp, group=64, n_grid=4)
+    for k in range(4):
+        _, _, _, w_hat = orc.quantize_weights_group_asym(w, res["scales"][k], 64)
+        dw = orc.bf16_to_f64(orc.delta_weights_bf16(w, w_hat))
+        exact = orc.bf16_to_f64(w) - w_hat.astype(np.float64)
+        assert np.all(np.abs(dw - exact) <= 2.0 ** -8 * np.abs(exact) + 1e-30)
+        e = ((orc.bf16_to_f64(x) @ dw.T) ** 2).sum(axis=1)
+        assert np.allclose(e, res["per_token"][k], rtol=5e-3)
+
+
+@pytest.mark.parametrize("mode", ["w8a8", "w4a8", "w4a6"])
+def test_apply_layer_symmetric_modes_with_bias(mode):
+    """f_q = Q_w(W scale) Q_a(x / scale) + b in the symmetric settings, against scalar loops over the integer codes:
+    the bias is added per output channel after the two steps have rescaled the integer product, it cancels in the
+    search error, and the quantizer outputs returned are those of the candidate."""
+    x, w, imp = wl.small_case(191, 7, 16, 5)
+    wn, an = orc.symmetric_bits(mode)
+    s = orc.scale_table(orc.channel_stat(x), 4)[2]
+    bias_bits = bits(np.array([0.5, -1.0, 0.0, 2.0, -0.25]))
+    b = orc.bf16_to_f64(bias_bits)
+    yq, (qw, u, none) = orc.apply_layer(x, w, s, bias_bits, mode)
+    assert none is None and yq.shape == (7, 5)
+    qw_ref, u_ref = orc.quantize_weights_row_sym(w, s, wn)
+    qx, t = orc.quantize_activations_token_sym(x, s, an)
+    assert np.array_equal(qw, qw_ref) and np.array_equal(u, u_ref)
+    for n in range(7):
+        for o in range(5):
+            acc = 0
+            for c in range(16):
+                acc += int(qx[n, c]) * int(qw[o, c])
+            assert math.isclose(yq[n, o], float(t[n]) * float(u[o]) * acc + float(b[o]), rel_tol=1e-13, abs_tol=1e-15)
+    # layer_q_w8a8 alone: bias per output channel (second axis), nothing else changes
+    y0 = orc.layer_q_w8a8(qx, t, qw, u)
+    y1 = orc.layer_q_w8a8(qx, t, qw, u, b)
+    assert np.allclose(y1 - y0, np.broadcast_to(b[None, :], (7, 5)), rtol=0, atol=1e-15)
+    # the bias cancels in the search error
+    e = orc.per_token_error(orc.layer_fp(x, w, b), yq)
+    assert np.allclose(e, orc.candidate_error(x, w, s, mode, 0), rtol=1e-9)
+    # without a scale the activations are quantized as they are
+    yq_plain, _ = orc.apply_layer(x, w, None, None, mode)
+    qx0, t0 = orc.quantize_sym_rows(orc.bf16_to_f64(x).astype(np.float32), an)
+    qw0, u0 = orc.quantize_weights_row_sym(w, None, wn)
+    assert np.allclose(yq_plain, orc.layer_q_w8a8(qx0, t0, qw0, u0), rtol=0, atol=0)
+
+
+def _search_with_exact_division(x, w, imp, group, n_grid):
+    """The group-mode search with the other reading of diag(scale)^-1 in the smoothing identity of Sec. 2.2: the
+    dequantized weight divided by the scale in one IEEE binary32 division, where the oracle multiplies by the
+    rounded reciprocal.  Codes, steps and zero-points are the oracle's (they do not depend on the reading)."""
+    scales = orc.scale_table(orc.channel_stat(x), n_grid)
+    y_fp = orc.layer_fp(x, w)
+    losses, per_token, ints = [], [], []
+    for k in range(n_grid):
+        codes, step, zero, _ = orc.quantize_weights_group_asym(w, scales[k], group)
+        c2, c1 = codes.shape
+        dq = ((codes.astype(np.int64).reshape(c2, c1 // group, group) - zero[:, :, None]).astype(np.float32)
+              * step[:, :, None]).astype(np.float32).reshape(c2, c1)
+        w_hat = (dq / scales[k][None, :].astype(np.float32)).astype(np.float32)
+        e = orc.per_token_error(y_fp, orc.layer_q_w4a16(x, w_hat))
+        per_token.append(e)
+        losses.append(orc.weighted_loss(e, imp, c2))
+        ints.append((codes, step, zero))
+    return np.array(losses), np.array(per_token), ints
+
+
+@pytest.mark.parametrize("shape", ["cfg0", (300, 192, 320, 64, 5), (515, 1088, 777, 64, 7), (128, 64, 256, 32, 3)])
+def test_reciprocal_and_division_readings_give_the_same_search(shape):
+    """Sec. 2.2 writes the smoothing as diag(scale)^-1; the oracle takes that as a product with the binary32
+    reciprocal (the same factor that smooths the activations).  Dividing by the scale instead changes W_hat by at
+    most an ulp, so the integers are untouched and every loss moves by far less than the stated tolerance; the
+    argmin is the same."""
+    if shape == "cfg0":
+        cfgw = wl.config("cfg0")
+        data = wl.LayerData(cfgw)
+        lin = cfgw.linear("q")
+        x, w, imp, group, n_grid = data.x(lin), data.w(lin), data.imp(), cfgw.group, cfgw.n_grid
+    else:
+        n, c1, c2, group, n_grid = shape
+        x, w, imp = wl.small_case(17, n, c1, c2, n_outlier=2)
+    ref = orc.scale_search(x, w, imp, "w4a16", group, n_grid)
+    losses, per_token, ints = _search_with_exact_division(x, w, imp, group, n_grid)
+    assert np.max(np.abs(losses - ref["losses"]) / ref["losses"]) < 1e-6
+    assert np.allclose(per_token, ref["per_token"], rtol=1e-5)
+    assert orc.argmin_lowest(losses) == ref["best"]
+    # the reading cannot reach the integers: they are computed before any division by the scale
+    for k in (0, n_grid - 1):
+        codes, step, zero, _ = orc.quantize_weights_group_asym(w, ref["scales"][k], group)
+        assert np.array_equal(codes, ints[k][0]) and np.array_equal(step, ints[k][1]) and np.array_equal(zero, ints[k][2])
+
+
+def test_reciprocal_and_division_readings_symmetric_activations():
+    """For quantized activations the reading reaches an integer decision: x * fl32(1/scale) against fl32(x / scale)
+    differ by an ulp in about a quarter of the elements, which moves a code only when the quotient sits within
+    that ulp of a rounding boundary.  Counted here: a few codes in a hundred thousand, losses equal to 1e-4."""
+    x, w, imp = wl.small_case(43, 256, 512, 512, n_outlier=2)
+    scales = orc.scale_table(orc.channel_stat(x), 20)
+    y_fp = orc.layer_fp(x, w)
+    xv = orc.bf16_to_f64(x).astype(np.float32)
+    flipped, total = 0, 0
+    for k in (5, 12, 19):
+        qx, t = orc.quantize_activations_token_sym(x, scales[k], 8)
+        qx_div, t_div = orc.quantize_sym_rows((xv / scales[k][None, :]).astype(np.float32), 8)
+        flipped += int((qx != qx_div).sum())
+        total += qx.size
+        assert np.max(np.abs(qx.astype(np.int64) - qx_div.astype(np.int64))) <= 1
+        qw, u = orc.quantize_weights_row_sym(w, scales[k], 8)
+        l_mul = orc.weighted_loss(orc.per_token_error(y_fp, orc.layer_q_w8a8(qx, t, qw, u)), imp, 512)
+        l_div = orc.weighted_loss(orc.per_token_error(y_fp, orc.layer_q_w8a8(qx_div, t_div, qw, u)), imp, 512)
+        assert abs(l_mul - l_div) / l_mul < 1e-4
+    assert flipped / total < 1e-3
