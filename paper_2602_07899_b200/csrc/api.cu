@@ -11,6 +11,17 @@ namespace tlq {
 
 long long g_launch_count = 0;
 
+int device_sm_count() {
+  static int sms[kMaxDevices] = {};
+  const int dev = current_device_index();
+  if (dev < 0) return 0;
+  if (sms[dev] == 0 && cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+    cudaGetLastError();
+    sms[dev] = 0;
+  }
+  return sms[dev];
+}
+
 namespace {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }

@@ -25,6 +25,33 @@ inline int after_launch() {
   return cudaGetLastError() == cudaSuccess ? TLQ_OK : TLQ_ERR_CUDA;
 }
 
+// Host-side state that belongs to a device (kernel attributes, SM counts) is kept per device index: one process
+// may drive several GPUs, each call acting on the device that is current when it is made.
+constexpr int kMaxDevices = 64;
+inline int current_device_index() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+  return dev;
+}
+int device_sm_count();   // multiprocessors of the current device (looked up once per device); 0 on error
+struct OncePerDevice {
+  bool done[kMaxDevices] = {};
+};
+// Runs `configure` (returning a cudaError_t) the first time it is reached with a given device current.
+template <typename F>
+inline int once_per_device(OncePerDevice& state, F configure) {
+  const int dev = current_device_index();
+  if (dev < 0) return TLQ_ERR_CUDA;
+  if (!state.done[dev]) {
+    if (configure() != cudaSuccess) {
+      cudaGetLastError();
+      return TLQ_ERR_CUDA;
+    }
+    state.done[dev] = true;
+  }
+  return TLQ_OK;
+}
+
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 

@@ -404,19 +404,20 @@ int launch_fakequant_group(const uint16_t* W, const uint16_t* s, const float* rs
   const bool hot = dW != nullptr && s != nullptr && rs != nullptr && codes == nullptr && steps == nullptr && zeros == nullptr;
   const int tile_rows = hot ? kHotRows : kGqRows;
   const int64_t ctas = ceil_div(C1, kGqCols) * ceil_div(C2, tile_rows);
-  int64_t kchunks = ceil_div(148 * 6, ctas);        // aim for several CTAs per SM
+  const int sms = device_sm_count();
+  if (sms <= 0) return TLQ_ERR_CUDA;
+  int64_t kchunks = ceil_div((int64_t)sms * 6, ctas);        // aim for several CTAs per SM
   if (kchunks > K) kchunks = K;
   if (kchunks < 1) kchunks = 1;
   const int k_per_cta = (int)ceil_div(K, kchunks);
   kchunks = ceil_div(K, k_per_cta);
   dim3 grid((unsigned)(ceil_div(C1, kGqCols) * ceil_div(C2, tile_rows)), (unsigned)kchunks);
   if (hot) {
-    static bool configured = false;
-    if (!configured) {
-      TLQ_CUDA_TRY(cudaFuncSetAttribute(fakequant_delta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)kHotSmem));
-      configured = true;
-    }
+    static OncePerDevice once;
+    const int rc_cfg = once_per_device(once, [] {
+      return cudaFuncSetAttribute(fakequant_delta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kHotSmem);
+    });
+    if (rc_cfg != TLQ_OK) return rc_cfg;
     // |quotient| <= qmax + 1 on the straight-line path; 4e-7 per unit covers the reciprocal (1 ulp), the product
     // and the exact quotient's own rounding (together < 2.4e-7 relative)
     const float tie_eps = 4.0e-7f * (float)(1 << w_bits);
@@ -638,16 +639,19 @@ row_codes_kernel(const uint16_t* __restrict__ src, const uint16_t* __restrict__ 
 }
 
 template <int kKind>
-static int launch_rows(const uint16_t* src, const uint16_t* s, const float* rs, int K, int64_t R, int64_t C1, int bits,
+static int launch_rows_two_pass(const uint16_t* src, const uint16_t* s, const float* rs, int K, int64_t R, int64_t C1, int bits,
                        int8_t* q, float* step, const int32_t* n_rows_dev, cudaStream_t st) {
-  static bool configured = false;      // one flag per instantiation of this template
-  if (!configured) {
-    TLQ_CUDA_TRY(cudaFuncSetAttribute(row_amax_kernel<kKind>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kRowSmem));
-    TLQ_CUDA_TRY(cudaFuncSetAttribute(row_codes_kernel<kKind>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kRowSmem));
-    configured = true;
-  }
+  static OncePerDevice once;      // one per instantiation of this template
+  int rc = once_per_device(once, [] {
+    const cudaError_t e = cudaFuncSetAttribute(row_amax_kernel<kKind>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kRowSmem);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(row_codes_kernel<kKind>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kRowSmem);
+  });
+  if (rc != TLQ_OK) return rc;
+  const int sms = device_sm_count();
+  if (sms <= 0) return TLQ_ERR_CUDA;
   const int64_t ctas = ceil_div(C1, kGqCols) * ceil_div(R, kRowRows);
-  int64_t kchunks = ceil_div(148 * 6, ctas);
+  int64_t kchunks = ceil_div((int64_t)sms * 6, ctas);
   if (kchunks > K) kchunks = K;
   if (kchunks < 1) kchunks = 1;
   const int k_per_cta = (int)ceil_div(K, kchunks);
@@ -659,12 +663,225 @@ static int launch_rows(const uint16_t* src, const uint16_t* s, const float* rs, 
   TLQ_CUDA_TRY(cudaMemsetAsync(step, 0, (size_t)n * sizeof(float), st));
   row_amax_kernel<kKind><<<grid, kGqThreads, kRowSmem, st>>>(src, s, rs, K, k_per_cta, R, n_rows_dev, C1,
                                                       reinterpret_cast<int*>(step));
-  int rc = after_launch();
+  rc = after_launch();
   if (rc != TLQ_OK) return rc;
   amax_to_step_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(step, n, qpos);
   if ((rc = after_launch()) != TLQ_OK) return rc;
   row_codes_kernel<kKind><<<grid, kGqThreads, kRowSmem, st>>>(src, s, rs, step, K, k_per_cta, R, n_rows_dev, C1, qpos, tie_eps, q);
   return after_launch();
+}
+
+// ------------------------------------------------------------------------------------------------
+// The same quantizer with whole rows resident in one CTA: one launch instead of four, the source read
+// from HBM once, and per element about half the instructions of the two tiled passes above.
+//
+// A CTA stages RB complete rows in shared memory (RB x C1 bf16, at most ~100 KB so that two CTAs share
+// an SM) and walks its candidates in order.  A thread owns fixed 16-channel columns, so the candidate's
+// per-channel multipliers are loaded once per column and serve all RB rows.  While the codes of
+// candidate k are formed, the same unpacked values are multiplied by candidate k+1's multipliers and
+// folded into running row maxima; the maxima are combined across the CTA (shuffles, then one warp per
+// row), which yields step and 1/step of candidate k+1 for the next round.  Only the first candidate of
+// a CTA needs a maximum pass of its own.  Per (row, candidate) the result is what the tiled passes
+// give: max over channels of |value| is taken over the same binary32 products, the step is the same
+// IEEE division, the codes come from the same straight-line arithmetic with the exact-division fix-up.
+// ------------------------------------------------------------------------------------------------
+constexpr int kFusedThreads = 256;
+constexpr int kFusedWarps = kFusedThreads / 32;
+constexpr size_t kFusedSmemBudget = 100 << 10;     // two CTAs per SM
+constexpr size_t kFusedSmemLimit = 220 << 10;      // one CTA per SM: the widest row this kernel takes
+
+template <int kKind, int RB>
+__global__ void __launch_bounds__(kFusedThreads, 2)
+row_quant_fused_kernel(const uint16_t* __restrict__ src, const uint16_t* __restrict__ s_tab,
+                       const float* __restrict__ rs_tab, int K, int k_per_cta, int64_t R_all,
+                       const int32_t* __restrict__ n_rows_dev, int64_t C1, float qpos, float tie_eps,
+                       int8_t* __restrict__ q /*[K,R_all,C1]*/, float* __restrict__ step /*[K,R_all]*/) {
+  extern __shared__ uint4 tile_dyn[];                 // [RB][C1 / 8]
+  __shared__ float red[2][kFusedWarps][RB];           // per-warp row maxima of the candidate being prepared
+  __shared__ float2 step_inv[2][RB];                  // (step, ~1/step) per row, double-buffered over candidates
+  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+  const int64_t R = (n_rows_dev != nullptr) ? (int64_t)*n_rows_dev : R_all;    // rows beyond are not live
+  const int64_t row0 = (int64_t)blockIdx.x * RB;
+  if (row0 >= R) return;                              // the whole CTA leaves together
+  const int nchunks = (int)(C1 >> 4);                 // 16-channel columns of a row
+  const int row_u4 = nchunks * 2;                     // uint4 per staged row
+  const int k_begin = blockIdx.y * k_per_cta;
+  const int k_end = min(K, k_begin + k_per_cta);
+
+  for (int i = t; i < RB * row_u4; i += kFusedThreads) {
+    const int r = i / row_u4, c = i - r * row_u4;
+    uint4 v = make_uint4(0, 0, 0, 0);                 // rows past the end count as zeros and store nothing
+    if (row0 + r < R) v = ld_nc_16(src + (row0 + r) * C1 + (int64_t)c * 8);
+    tile_dyn[i] = v;
+  }
+  // Narrow rows leave threads over: they are dealt out over row groups, thread (rg, column) taking rows rg, rg + groups, ...
+  const int col_threads = nchunks < kFusedThreads ? nchunks : kFusedThreads;
+  const int groups = kFusedThreads / col_threads;
+  const int rg = t / col_threads;
+  const int col0 = t - rg * col_threads;
+  uint32_t row_mask = 0;
+  if (rg < groups)
+    for (int r = rg; r < RB; r += groups) row_mask |= 1u << r;
+  __syncthreads();
+
+  const float tie_lim = 0.5f - tie_eps;
+  const float2 magic2 = make_float2(kMagic, kMagic);
+  auto mult_rows = [&](int k, const uint16_t*& s_row, const float*& rs_row) {
+    s_row = s_tab ? s_tab + (int64_t)k * C1 : nullptr;
+    rs_row = rs_tab ? rs_tab + (int64_t)k * C1 : nullptr;
+  };
+  // Combine the threads' running maxima of candidate k into (step, 1/step) per row; buffer `par`.
+  auto publish = [&](float (&am)[RB], int par, int k) {
+#pragma unroll
+    for (int r = 0; r < RB; ++r) {
+      float v = am[r];
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, off));
+      if (lane == 0) red[par][warp][r] = v;
+    }
+    __syncthreads();
+    if (warp < RB) {                                  // warp w finishes row w
+      float v = lane < kFusedWarps ? red[par][lane][warp] : 0.0f;
+#pragma unroll
+      for (int off = kFusedWarps / 2; off > 0; off >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, off));
+      if (lane == 0) {
+        const float st = __fdiv_rn(fmaxf(v, TLQ_RANGE_FLOOR), qpos);
+        step_inv[par][warp] = make_float2(st, rcp_fast(st));
+        if (row0 + warp < R) step[(int64_t)k * R_all + row0 + warp] = st;
+      }
+    }
+    __syncthreads();
+  };
+
+  float am[RB];
+#pragma unroll
+  for (int r = 0; r < RB; ++r) am[r] = 0.0f;
+  if (row_mask != 0) {                                // the first candidate's maxima: a pass of its own
+    const uint16_t* s_row; const float* rs_row;
+    mult_rows(k_begin, s_row, rs_row);
+    for (int ch = col0; ch < nchunks; ch += col_threads) {
+      float2 m[8];
+      load_mult16<kKind>(s_row, rs_row, (int64_t)ch * 16, true, m);
+#pragma unroll
+      for (int r = 0; r < RB; ++r) {
+        if (!((row_mask >> r) & 1u)) continue;
+        float2 w[8];
+        unpack16(tile_dyn[r * row_u4 + ch * 2], tile_dyn[r * row_u4 + ch * 2 + 1], w);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const float2 v = mul2(w[j], m[j]);
+          am[r] = max3(am[r], fabsf(v.x), fabsf(v.y));
+        }
+      }
+    }
+  }
+  publish(am, 0, k_begin);
+
+  for (int k = k_begin; k < k_end; ++k) {
+    const int par = (k - k_begin) & 1;
+    const bool has_next = k + 1 < k_end;
+    float st[RB], inv[RB];
+#pragma unroll
+    for (int r = 0; r < RB; ++r) {
+      const float2 si = step_inv[par][r];
+      st[r] = si.x; inv[r] = si.y;
+      am[r] = 0.0f;
+    }
+    if (row_mask != 0) {
+      const uint16_t* s_row; const float* rs_row;
+      const uint16_t* s_next = nullptr; const float* rs_next = nullptr;
+      mult_rows(k, s_row, rs_row);
+      if (has_next) mult_rows(k + 1, s_next, rs_next);
+      for (int ch = col0; ch < nchunks; ch += col_threads) {
+        float2 m[8], m2[8];
+        load_mult16<kKind>(s_row, rs_row, (int64_t)ch * 16, true, m);
+        if (has_next) load_mult16<kKind>(s_next, rs_next, (int64_t)ch * 16, true, m2);
+#pragma unroll
+        for (int r = 0; r < RB; ++r) {
+          if (!((row_mask >> r) & 1u)) continue;
+          const uint4* tile16 = &tile_dyn[r * row_u4 + ch * 2];
+          float2 w[8];
+          unpack16(tile16[0], tile16[1], w);
+          if (has_next) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const float2 v = mul2(w[j], m2[j]);
+              am[r] = max3(am[r], fabsf(v.x), fabsf(v.y));
+            }
+          }
+          const int64_t row = row0 + r;
+          if (row >= R) continue;
+          const float2 inv2 = make_float2(inv[r], inv[r]);
+          float near = 0.0f;
+          uint32_t tb[16];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const float2 qv = mul2(mul2(w[j], m[j]), inv2);
+            const float2 tt = add2(qv, magic2);          // low mantissa byte = the code in two's complement
+            const float2 df = sub2(qv, sub2(tt, magic2));
+            near = max3(near, fabsf(df.x), fabsf(df.y));
+            tb[2 * j] = __float_as_uint(tt.x);
+            tb[2 * j + 1] = __float_as_uint(tt.y);
+          }
+          uint4* dst = reinterpret_cast<uint4*>(q + ((int64_t)k * R_all + row) * C1 + (int64_t)ch * 16);
+          if (near > tie_lim) {
+            float mf[16];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { mf[2 * j] = m[j].x; mf[2 * j + 1] = m[j].y; }
+            codes16_exact(tile16, mf, st[r], qpos, dst);
+          } else {
+            uint32_t pk[4];
+#pragma unroll
+            for (int g = 0; g < 4; ++g)
+              pk[g] = __byte_perm(__byte_perm(tb[4 * g], tb[4 * g + 1], 0x0040),
+                                  __byte_perm(tb[4 * g + 2], tb[4 * g + 3], 0x0040), 0x5410);
+            *dst = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          }
+        }
+      }
+    }
+    if (has_next) publish(am, par ^ 1, k + 1);
+  }
+}
+
+template <int kKind, int RB>
+static int launch_rows_fused(const uint16_t* src, const uint16_t* s, const float* rs, int K, int64_t R, int64_t C1,
+                             int bits, int8_t* q, float* step, const int32_t* n_rows_dev, cudaStream_t st) {
+  static OncePerDevice once;
+  int rc = once_per_device(once, [] {
+    return cudaFuncSetAttribute(row_quant_fused_kernel<kKind, RB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)kFusedSmemLimit);
+  });
+  if (rc != TLQ_OK) return rc;
+  const int sms = device_sm_count();
+  if (sms <= 0) return TLQ_ERR_CUDA;
+  const int64_t row_blocks = ceil_div(R, RB);
+  int64_t kchunks = ceil_div((int64_t)sms * 12, row_blocks);     // several work units per resident CTA
+  if (kchunks > K) kchunks = K;
+  if (kchunks < 1) kchunks = 1;
+  const int k_per_cta = (int)ceil_div(K, kchunks);
+  kchunks = ceil_div(K, k_per_cta);
+  const dim3 grid((unsigned)row_blocks, (unsigned)kchunks);
+  const float qpos = (float)((1 << (bits - 1)) - 1);
+  const float tie_eps = 4.0e-7f * (qpos + 1.0f);
+  const size_t smem = (size_t)RB * (size_t)C1 * 2;
+  row_quant_fused_kernel<kKind, RB><<<grid, kFusedThreads, smem, st>>>(src, s, rs, K, k_per_cta, R, n_rows_dev, C1, qpos,
+                                                                  tie_eps, q, step);
+  return after_launch();
+}
+
+// Rows per CTA of the whole-row kernel: the largest of 8, 4, 2, 1 whose rows fit the shared-memory budget; rows too
+// wide even for one per CTA go through the two tiled passes.
+template <int kKind>
+static int launch_rows(const uint16_t* src, const uint16_t* s, const float* rs, int K, int64_t R, int64_t C1, int bits,
+                       int8_t* q, float* step, const int32_t* n_rows_dev, cudaStream_t st) {
+  const size_t row_bytes = (size_t)C1 * 2;
+  if ((C1 & 15) != 0 || row_bytes > kFusedSmemLimit)
+    return launch_rows_two_pass<kKind>(src, s, rs, K, R, C1, bits, q, step, n_rows_dev, st);
+  if (8 * row_bytes <= kFusedSmemBudget) return launch_rows_fused<kKind, 8>(src, s, rs, K, R, C1, bits, q, step, n_rows_dev, st);
+  if (4 * row_bytes <= kFusedSmemBudget) return launch_rows_fused<kKind, 4>(src, s, rs, K, R, C1, bits, q, step, n_rows_dev, st);
+  if (2 * row_bytes <= kFusedSmemBudget) return launch_rows_fused<kKind, 2>(src, s, rs, K, R, C1, bits, q, step, n_rows_dev, st);
+  return launch_rows_fused<kKind, 1>(src, s, rs, K, R, C1, bits, q, step, n_rows_dev, st);
 }
 
 int launch_fakequant_rows_i8(const uint16_t* W, const uint16_t* s, int K, int64_t C2, int64_t C1, int bits, int8_t* q,

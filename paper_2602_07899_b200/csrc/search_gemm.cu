@@ -270,25 +270,14 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   }
 }
 
-int num_sms() {
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) sms = 0;
-  }
-  return sms;
-}
+int num_sms() { return device_sm_count(); }
 
 template <bool kApply>
 int configure_kernel() {
-  static bool done = false;
-  if (!done) {
-    TLQ_CUDA_TRY(cudaFuncSetAttribute(gemm_bf16_kernel<kApply>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      (int)kSmemBytes));
-    done = true;
-  }
-  return TLQ_OK;
+  static OncePerDevice once;
+  return once_per_device(once, [] {
+    return cudaFuncSetAttribute(gemm_bf16_kernel<kApply>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+  });
 }
 
 }  // namespace

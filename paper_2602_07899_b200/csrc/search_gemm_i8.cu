@@ -386,25 +386,14 @@ gemm_w8a8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
   }
 }
 
-int sm_count() {
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) sms = 0;
-  }
-  return sms;
-}
+int sm_count() { return device_sm_count(); }
 
 template <int kMode>
 int configure_kernel() {
-  static bool done = false;
-  if (!done) {
-    TLQ_CUDA_TRY(cudaFuncSetAttribute(gemm_w8a8_kernel<kMode>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      (int)kSmemBytes));
-    done = true;
-  }
-  return TLQ_OK;
+  static OncePerDevice once;
+  return once_per_device(once, [] {
+    return cudaFuncSetAttribute(gemm_w8a8_kernel<kMode>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+  });
 }
 
 bool map_bf16_2d(CUtensorMap* tm, const uint16_t* p, int64_t rows, int64_t C1, uint32_t box_rows) {

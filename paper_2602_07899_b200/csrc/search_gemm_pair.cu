@@ -237,8 +237,12 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
 }
 
 int max_pairs() {
-  static int pairs = -1;
-  if (pairs < 0) {
+  static int pairs_of[kMaxDevices];
+  static bool known[kMaxDevices] = {};
+  const int dev = current_device_index();
+  if (dev < 0) return 0;
+  int& pairs = pairs_of[dev];
+  if (!known[dev]) {
     if (cudaFuncSetAttribute(gemm_bf16_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) !=
         cudaSuccess)
       return 0;
@@ -257,6 +261,7 @@ int max_pairs() {
       return 0;
     }
     pairs = n;
+    known[dev] = true;
   }
   return pairs;
 }

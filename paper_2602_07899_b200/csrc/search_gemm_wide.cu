@@ -231,27 +231,18 @@ gemm_bf16_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
   }
 }
 
-int wide_sm_count() {
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) sms = 0;
-  }
-  return sms;
-}
+int wide_sm_count() { return device_sm_count(); }
 
 }  // namespace
 
 int launch_search_gemm_bf16_wide(const uint16_t* X, const uint16_t* dW, const float* w_imp, const GemmPlan& plan,
                                  float* partials, float* ptab, WorkspaceHeader* hdr, const int32_t* n_live,
                                  cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
-    TLQ_CUDA_TRY(cudaFuncSetAttribute(gemm_bf16_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      (int)kSmemBytes));
-    configured = true;
-  }
+  static OncePerDevice once;
+  const int rc_cfg = once_per_device(once, [] {
+    return cudaFuncSetAttribute(gemm_bf16_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+  });
+  if (rc_cfg != TLQ_OK) return rc_cfg;
   CUtensorMap tmA, tmB;
   const uint64_t adims[2] = {(uint64_t)plan.C1, (uint64_t)plan.N};
   const uint64_t astr[1] = {(uint64_t)plan.C1 * 2};

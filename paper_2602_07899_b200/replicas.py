@@ -84,18 +84,30 @@ def shard_rows(c_out: int, info: RankInfo) -> Tuple[int, int]:
     return row0, row0 + base + (1 if info.rank < extra else 0)
 
 
-def combine_sharded_losses(local_losses: torch.Tensor, local_rows: int, c_out: int, info: RankInfo):
-    """Losses of the whole matrix from the ranks' slice losses (each normalised by its own row count, as the
-    search returns them): sum_r rows_r * loss_r / c_out.  Returns (losses float64 [K], argmin with the lowest
-    index on ties).  `local_losses` may live on the GPU (NCCL) or the CPU (gloo)."""
-    t = local_losses.to(torch.float64) * float(local_rows)
-    if info.world > 1:
-        t = t.clone()
-        dist.all_reduce(t, op=dist.ReduceOp.SUM)
-    total = t / float(c_out)
+def weighted_slice_losses(local_losses: torch.Tensor, local_rows: int) -> torch.Tensor:
+    """A slice's losses (normalised by its own row count, as the search returns them) turned back into sums over
+    its rows: what the ranks add up."""
+    return local_losses.to(torch.float64) * float(local_rows)
+
+
+def finish_sharded_losses(summed: torch.Tensor, c_out: int):
+    """Losses of the whole matrix from the sum of the slices' weighted losses, and the argmin with the lowest
+    index on ties.  Returns (losses float64 [K], argmin)."""
+    total = summed / float(c_out)
     vals = total.cpu().tolist()
     best, bv = 0, float("inf")
     for k, v in enumerate(vals):
         if v < bv:
             best, bv = k, v
     return total, best
+
+
+def combine_sharded_losses(local_losses: torch.Tensor, local_rows: int, c_out: int, info: RankInfo):
+    """Losses of the whole matrix from the ranks' slice losses: sum_r rows_r * loss_r / c_out, one SUM reduction of
+    K doubles.  Returns (losses float64 [K], argmin with the lowest index on ties).  `local_losses` may live on the
+    GPU (NCCL) or the CPU (gloo)."""
+    t = weighted_slice_losses(local_losses, local_rows)
+    if info.world > 1:
+        t = t.clone()
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return finish_sharded_losses(t, c_out)

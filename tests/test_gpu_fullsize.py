@@ -24,6 +24,15 @@ def tlq():
     return mod
 
 
+def assert_same_argmin(best, ref, floor=1e-4):
+    """No argmin but the oracle's is accepted; that the oracle's own two best candidates are far enough apart for
+    this to be a fair demand is asserted on the seeded data first."""
+    order = np.sort(ref["losses"])
+    gap = (order[1] - order[0]) / order[0]
+    assert gap > floor, f"the oracle's top-2 gap is {gap:.2e}: ambiguous seeded case"
+    assert best == ref["best"]
+
+
 def bits_of(t):
     return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
 
@@ -64,9 +73,7 @@ def full_compare(tlq, cfgw, lin_name):
     got = gpu_search(tlq, cfgw, xb, wb, imp)
     np.testing.assert_allclose(got["per_token"], ref["per_token"], rtol=LOSS_RTOL, atol=1e-30)
     np.testing.assert_allclose(got["losses"], ref["losses"], rtol=LOSS_RTOL)
-    order = np.sort(ref["losses"])
-    if (order[1] - order[0]) / order[0] > 1e-5:
-        assert got["best"] == ref["best"]
+    assert_same_argmin(got["best"], ref)
     assert np.array_equal(got["s_best"], orc.f32_to_bf16_bits(ref["scales"][got["best"]]))
     check_properties(got, imp, lin.c_out)
     return ref, got
@@ -169,9 +176,7 @@ def test_7b_k_projection_full_paper_settings(tlq):
     cfg = tlq.config(tlq.WA_SYM_CHANNEL, w_bits=4, a_bits=8, n_grid=cfgw.n_grid, flags=tlq.FLAG_SKIP_ZERO_WEIGHT_TOKENS)
     out = tlq.tlq_scale_search_layer(tlq.bf16_from_bits(xb), tlq.bf16_from_bits(wb), torch.from_numpy(mask).cuda(), cfg)
     np.testing.assert_allclose(out.losses.cpu().numpy(), ref["losses"], rtol=LOSS_RTOL)
-    order = np.sort(ref["losses"])
-    if (order[1] - order[0]) / order[0] > 1e-5:
-        assert int(out.best_idx.item()) == ref["best"]
+    assert_same_argmin(int(out.best_idx.item()), ref)
 
 
 @pytest.mark.parametrize("key", ["cfg1", "cfg2"])
@@ -191,6 +196,4 @@ def test_7b_k_projection_full_two_streams(tlq, key):
                                      per_token=True, X_fp=tlq.bf16_from_bits(xf))
     np.testing.assert_allclose(out.per_token.cpu().numpy(), ref["per_token"], rtol=LOSS_RTOL, atol=1e-30)
     np.testing.assert_allclose(out.losses.cpu().numpy(), ref["losses"], rtol=LOSS_RTOL)
-    order = np.sort(ref["losses"])
-    if (order[1] - order[0]) / order[0] > 1e-5:
-        assert int(out.best_idx.item()) == ref["best"]
+    assert_same_argmin(int(out.best_idx.item()), ref)
