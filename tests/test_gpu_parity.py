@@ -689,8 +689,9 @@ def test_row_sharded_search_combines_to_the_unsharded_result(tlq, mode):
     assert_same_argmin(best, ref)
 
 
-def test_row_quantizers_for_rows_wider_than_one_cta_can_hold(tlq):
-    """Rows too wide for the whole-row kernel's shared memory go through the two tiled passes: same contract."""
+def test_row_quantizers_on_very_wide_rows(tlq):
+    """A few rows of more than a hundred thousand channels (224 column tiles per row, every row maximum combined
+    from that many partial maxima): same contract."""
     c1 = 114688
     xb = wl.activations(191, "wide/x", 6, c1, 4, "normal", 4)
     wb = wl.weights(191, "wide/w", 5, c1)
