@@ -226,6 +226,17 @@ int tlq_apply_layer(const void* X, int64_t N, int64_t C1, const void* W, int64_t
 int tlq_read_status(const void* workspace, void* stream);
 
 /*
+ * Diagnostic of the device-side error path (the paper has no counterpart).  Every barrier wait inside the fused
+ * tensor-core kernels is bounded; when a bound expires the kernel writes TLQ_ERR_TIMEOUT to the status word and
+ * returns instead of hanging.  A correct run never gets there, so this call takes that path on purpose and
+ * harmlessly: one warp waits `limit_cycles` SM clock cycles (1 .. 2e9, i.e. at most about a second) on a barrier
+ * that nothing arrives on, then reports through the status word of `workspace` (at least 256 bytes, 16-byte
+ * aligned, zeroed by this call).  Afterwards tlq_read_status(workspace, stream) returns TLQ_ERR_TIMEOUT and the
+ * device context is as usable as before: no fault, no trap, no unbounded loop.
+ */
+int tlq_selftest_bounded_wait(void* workspace, size_t workspace_bytes, int64_t limit_cycles, void* stream);
+
+/*
  * Per-stage device timing of tlq_scale_search_layer, for benchmarks.  While enabled, every search call
  * records CUDA events on its stream between its stages (event sets come from a pool of 512 created on
  * first use; further calls are not recorded).  _drain() synchronises on the recorded events, writes

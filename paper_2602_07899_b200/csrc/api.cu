@@ -181,7 +181,7 @@ const char* tlq_status_string(int status) {
   }
 }
 
-int tlq_version(void) { return 1004; }   // 1.4: symmetric widths, flags, two-stream search, 4-bit packing
+int tlq_version(void) { return 1005; }   // 1.5: bounded-wait self-test
 
 int64_t tlq_kernel_launch_count(void) { return (int64_t)g_launch_count; }
 
@@ -478,6 +478,18 @@ int tlq_read_status(const void* workspace, void* stream) {
   int32_t status = 0;
   if (cudaMemcpy(&status, workspace, sizeof(status), cudaMemcpyDeviceToHost) != cudaSuccess) return TLQ_ERR_CUDA;
   return status;
+}
+
+int tlq_selftest_bounded_wait(void* workspace, size_t workspace_bytes, int64_t limit_cycles, void* stream) {
+  if (workspace == nullptr) return TLQ_ERR_INVALID_ARG;
+  if (!aligned16(workspace)) return TLQ_ERR_ALIGN;
+  if (workspace_bytes < sizeof(WorkspaceHeader)) return TLQ_ERR_WORKSPACE;
+  if (limit_cycles < 1 || limit_cycles > 2000000000LL) return TLQ_ERR_INVALID_ARG;   // at most about a second
+  int rc = have_device();
+  if (rc != TLQ_OK) return rc;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  TLQ_CUDA_TRY(cudaMemsetAsync(workspace, 0, sizeof(WorkspaceHeader), st));
+  return launch_bounded_wait_selftest(reinterpret_cast<WorkspaceHeader*>(workspace), (long long)limit_cycles, st);
 }
 
 int tlq_stage_timing_enable(int on) {

@@ -185,6 +185,9 @@ int launch_loss_reduce(const float* partials, int64_t per_k, int K, const float*
 int launch_per_token_reduce(const float* ptab /*[K,otiles,Npad]*/, int K, int64_t otiles, int64_t Npad, int64_t N,
                             float* per_token /*[K,N]*/, cudaStream_t st);
 
+// selftest.cu: one warp waits `limit_cycles` on a barrier nobody arrives on, then reports TLQ_ERR_TIMEOUT in `hdr`
+int launch_bounded_wait_selftest(WorkspaceHeader* hdr, long long limit_cycles, cudaStream_t st);
+
 // search_gemm.cu
 struct GemmPlan {
   int64_t N, C1, C2;

@@ -47,27 +47,53 @@ __device__ __forceinline__ float quotient_rint_clamped(float v, float step, floa
   return r;
 }
 
-// ---- packed binary32 pairs: one instruction carries two independent IEEE round-to-nearest operations
-__device__ __forceinline__ float2 mul2(float2 a, float2 b) {
-  float2 r;
-  asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
-      "mul.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
-      : "=f"(r.x), "=f"(r.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+// ---- packed binary32 pairs: one instruction carries two independent IEEE round-to-nearest operations.
+// A pair travels in ONE 64-bit register from its first use to its last: re-pairing two 32-bit registers around
+// every operation costs two moves per operand, more than the packed instruction saves (measured: 45 % of the
+// executed instructions of the row quantizers were such moves).
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pair_of(float lo, float hi) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
   return r;
 }
-__device__ __forceinline__ float2 add2(float2 a, float2 b) {
+__device__ __forceinline__ float2 halves(f32x2 v) {
   float2 r;
-  asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
-      "add.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
-      : "=f"(r.x), "=f"(r.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(r.x), "=f"(r.y) : "l"(v));
   return r;
 }
-__device__ __forceinline__ float2 sub2(float2 a, float2 b) {
-  float2 r;
-  asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
-      "sub.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
-      : "=f"(r.x), "=f"(r.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+__device__ __forceinline__ f32x2 pmul(f32x2 a, f32x2 b) {
+  f32x2 r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
   return r;
+}
+__device__ __forceinline__ f32x2 padd(f32x2 a, f32x2 b) {
+  f32x2 r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ f32x2 psub(f32x2 a, f32x2 b) {
+  f32x2 r;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+// two bf16 values packed in a 32-bit word -> their binary32 values as a pair (low half first)
+__device__ __forceinline__ f32x2 bf16x2_to_pair(uint32_t v) {
+  return pair_of(__uint_as_float(v << 16), __uint_as_float(v & 0xFFFF0000u));
+}
+__device__ __forceinline__ void unpack16_pairs(const uint4& t0, const uint4& t1, f32x2 (&w)[8]) {
+  w[0] = bf16x2_to_pair(t0.x); w[1] = bf16x2_to_pair(t0.y); w[2] = bf16x2_to_pair(t0.z); w[3] = bf16x2_to_pair(t0.w);
+  w[4] = bf16x2_to_pair(t1.x); w[5] = bf16x2_to_pair(t1.y); w[6] = bf16x2_to_pair(t1.z); w[7] = bf16x2_to_pair(t1.w);
+}
+// sixteen consecutive binary32 table entries (64-byte aligned) as eight pairs
+__device__ __forceinline__ void load_pairs16(const float* p, f32x2 (&m)[8]) {
+  const ulonglong2* q = reinterpret_cast<const ulonglong2*>(p);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const ulonglong2 v = q[j];
+    m[2 * j] = v.x;
+    m[2 * j + 1] = v.y;
+  }
 }
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float r;
@@ -79,11 +105,6 @@ __device__ __forceinline__ float min3(float a, float b, float c) {
   asm("min.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
   return r;
 }
-// two bf16 values packed in a 32-bit word -> their binary32 values (low half first)
-__device__ __forceinline__ float2 unpack2(uint32_t v) {
-  return make_float2(__uint_as_float(v << 16), __uint_as_float(v & 0xFFFF0000u));
-}
-
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
@@ -105,8 +126,6 @@ constexpr int kHotRows = 64;     // tile height of the delta-weight kernel: 64 K
 constexpr int kGqCols = 512;
 constexpr int kGqThreads = 256;
 constexpr size_t kHotSmem = (size_t)kHotRows * kGqCols * 2;
-constexpr int kRowRows = 32;     // row quantizers: 32 KB tiles leave the L1 to the per-candidate reciprocal tables (64-row tiles measured slower)
-constexpr size_t kRowSmem = (size_t)kRowRows * kGqCols * 2;
 
 // ------------------------------------------------------------------------------------------------
 // The search's own fake-quant pass: delta weights of ALL candidates, nothing else.  Same tile and
@@ -148,6 +167,88 @@ __device__ __noinline__ void delta16_general(const uint4* tile16, const uint16_t
   }
 }
 
+// What the head of a row leaves for its tail: the unpacked weights, the group's minimum, step and reciprocal, and
+// whether the group can clip.
+struct RowHead {
+  f32x2 w[8];
+  float mn, step, inv;
+  bool fast;
+};
+
+__device__ __forceinline__ void row_head(const uint4& t0, const uint4& t1, const f32x2 (&sv)[8], int lanes_per_group,
+                                         float qmax_f, float tie_lim, RowHead& h) {
+  unpack16_pairs(t0, t1, h.w);
+  float mx, mn;
+  {
+    const float2 p0 = halves(pmul(sv[0], h.w[0]));       // exact: 8-bit x 8-bit significands
+    mx = fmaxf(p0.x, p0.y);
+    mn = fminf(p0.x, p0.y);
+#pragma unroll
+    for (int j = 1; j < 8; ++j) {
+      const float2 pj = halves(pmul(sv[j], h.w[j]));
+      mx = max3(mx, pj.x, pj.y);
+      mn = min3(mn, pj.x, pj.y);
+    }
+  }
+  for (int off = 1; off < lanes_per_group; off <<= 1) {
+    mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
+    mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, off));
+  }
+  const float range = fmaxf(__fsub_rn(mx, mn), TLQ_RANGE_FLOOR);
+  const float step = __fdiv_rn(range, qmax_f);
+  const float inv = rcp_fast(step);
+  const float qa = __fmul_rn(mn, inv), qb = __fmul_rn(mx, inv);
+  float ra = round_magic(qa), rb = round_magic(qb);
+  if (fmaxf(fabsf(__fsub_rn(qa, ra)), fabsf(__fsub_rn(qb, rb))) > tie_lim) {
+    // an extreme sits on a rounding tie (common for bf16 weights: mx == -mn puts both on +-qmax/2): decide exactly
+    ra = round_magic(__fdiv_rn(mn, step));
+    rb = round_magic(__fdiv_rn(mx, step));
+  }
+  h.mn = mn; h.step = step; h.inv = inv;
+  h.fast = ra <= 0.0f && ra >= -qmax_f && __fsub_rn(rb, ra) <= qmax_f;   // the group cannot clip
+}
+
+__device__ __forceinline__ void row_tail(const RowHead& h, const f32x2 (&sv)[8], const f32x2 (&rsv)[8], float tie_lim,
+                                         float qmax_f, bool col_ok, const uint4* tile16, const uint16_t* s16,
+                                         const float* rs16, uint4* dst) {
+  if (!h.fast) {
+    if (col_ok) delta16_general(tile16, s16, rs16, h.mn, h.step, h.inv, qmax_f, dst);
+    return;
+  }
+  const f32x2 magic2 = pair_of(kMagic, kMagic);
+  const f32x2 inv2 = pair_of(h.inv, h.inv), step2 = pair_of(h.step, h.step);
+  uint32_t outw[8];
+  float near = 0.0f;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const f32x2 q = pmul(pmul(sv[j], h.w[j]), inv2);
+    const f32x2 rq = psub(padd(q, magic2), magic2);      // rint(q), which is q - z
+    const float2 df = halves(psub(q, rq));
+    near = max3(near, fabsf(df.x), fabsf(df.y));
+    const float2 d = halves(psub(h.w[j], pmul(pmul(rq, step2), rsv[j])));
+    outw[j] = pack_bf16x2(d.x, d.y);
+  }
+  if (near > tie_lim) {
+    // some element of this thread is near a tie: find the pair(s) and redo them with the exact quotient
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const f32x2 pr = pmul(sv[j], h.w[j]);
+      const f32x2 q = pmul(pr, inv2);
+      const float2 df = halves(psub(q, psub(padd(q, magic2), magic2)));
+      if (fmaxf(fabsf(df.x), fabsf(df.y)) > tie_lim) {
+        const float2 pj = halves(pr);
+        const f32x2 rq = pair_of(round_magic(__fdiv_rn(pj.x, h.step)), round_magic(__fdiv_rn(pj.y, h.step)));
+        const float2 d = halves(psub(h.w[j], pmul(pmul(rq, step2), rsv[j])));
+        outw[j] = pack_bf16x2(d.x, d.y);
+      }
+    }
+  }
+  if (col_ok) {
+    dst[0] = make_uint4(outw[0], outw[1], outw[2], outw[3]);
+    dst[1] = make_uint4(outw[4], outw[5], outw[6], outw[7]);
+  }
+}
+
 __global__ void __launch_bounds__(kGqThreads, 2)
 fakequant_delta_kernel(const uint16_t* __restrict__ W, const uint16_t* __restrict__ s_tab,
                        const float* __restrict__ rs_tab, int K, int k_per_cta, int64_t C2, int64_t C1, int group,
@@ -180,100 +281,24 @@ fakequant_delta_kernel(const uint16_t* __restrict__ W, const uint16_t* __restric
   }
   __syncthreads();
 
-  const float2 magic2 = make_float2(kMagic, kMagic);
   for (int k = k_begin; k < k_end; ++k) {
-    float2 sv[8], rsv[8];
+    f32x2 sv[8], rsv[8];
     if (!col_ok) {          // lanes past the last channel work on zeros and store nothing
 #pragma unroll
-      for (int j = 0; j < 8; ++j) sv[j] = rsv[j] = make_float2(1.0f, 1.0f);
+      for (int j = 0; j < 8; ++j) sv[j] = rsv[j] = pair_of(1.0f, 1.0f);
     } else {
       const uint4* sp = reinterpret_cast<const uint4*>(s_tab + (int64_t)k * C1 + c0);
-      const uint4 a = sp[0], b = sp[1];
-      sv[0] = unpack2(a.x); sv[1] = unpack2(a.y); sv[2] = unpack2(a.z); sv[3] = unpack2(a.w);
-      sv[4] = unpack2(b.x); sv[5] = unpack2(b.y); sv[6] = unpack2(b.z); sv[7] = unpack2(b.w);
-      const float4* rp = reinterpret_cast<const float4*>(rs_tab + (int64_t)k * C1 + c0);
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const float4 r4 = rp[j];
-        rsv[2 * j] = make_float2(r4.x, r4.y);
-        rsv[2 * j + 1] = make_float2(r4.z, r4.w);
-      }
+      unpack16_pairs(sp[0], sp[1], sv);
+      load_pairs16(rs_tab + (int64_t)k * C1 + c0, rsv);
     }
 #pragma unroll 1
     for (int p = 0; p < kHotRows / 8; ++p) {
       const int r = p * 8 + warp;
-      const int64_t row = row0 + r;
-      if (row >= C2) break;                       // rows of a warp ascend with p; shuffles below stay warp-uniform
-      const uint4 t0 = tile[r][lane * 2], t1 = tile[r][lane * 2 + 1];
-      float2 w[8];
-      w[0] = unpack2(t0.x); w[1] = unpack2(t0.y); w[2] = unpack2(t0.z); w[3] = unpack2(t0.w);
-      w[4] = unpack2(t1.x); w[5] = unpack2(t1.y); w[6] = unpack2(t1.z); w[7] = unpack2(t1.w);
-      float mx, mn;
-      {
-        const float2 p0 = mul2(sv[0], w[0]);       // exact: 8-bit x 8-bit significands
-        mx = fmaxf(p0.x, p0.y);
-        mn = fminf(p0.x, p0.y);
-#pragma unroll
-        for (int j = 1; j < 8; ++j) {
-          const float2 pj = mul2(sv[j], w[j]);
-          mx = max3(mx, pj.x, pj.y);
-          mn = min3(mn, pj.x, pj.y);
-        }
-      }
-      for (int off = 1; off < lanes_per_group; off <<= 1) {
-        mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
-        mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, off));
-      }
-      const float range = fmaxf(__fsub_rn(mx, mn), TLQ_RANGE_FLOOR);
-      const float step = __fdiv_rn(range, qmax_f);
-      const float inv = rcp_fast(step);
-      const float qa = __fmul_rn(mn, inv), qb = __fmul_rn(mx, inv);
-      float ra = round_magic(qa), rb = round_magic(qb);
-      if (fmaxf(fabsf(__fsub_rn(qa, ra)), fabsf(__fsub_rn(qb, rb))) > tie_lim) {
-        // an extreme sits on a rounding tie (common for bf16 weights: mx == -mn puts both on +-qmax/2): decide exactly
-        ra = round_magic(__fdiv_rn(mn, step));
-        rb = round_magic(__fdiv_rn(mx, step));
-      }
-      const bool fast = ra <= 0.0f && ra >= -qmax_f && __fsub_rn(rb, ra) <= qmax_f;   // the group cannot clip
-      uint32_t outw[8];
-      if (fast) {
-        const float2 inv2 = make_float2(inv, inv), step2 = make_float2(step, step);
-        float near = 0.0f;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const float2 pj = mul2(sv[j], w[j]);
-          const float2 q = mul2(pj, inv2);
-          const float2 rq = sub2(add2(q, magic2), magic2);      // rint(q), which is q - z
-          const float2 df = sub2(q, rq);
-          near = max3(near, fabsf(df.x), fabsf(df.y));
-          const float2 w_hat = mul2(mul2(rq, step2), rsv[j]);
-          const float2 d = sub2(w[j], w_hat);
-          outw[j] = pack_bf16x2(d.x, d.y);
-        }
-        if (near > tie_lim) {
-          // some element of this thread is near a tie: find the pair(s) and redo them with the exact quotient
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const float2 pj = mul2(sv[j], w[j]);
-            const float2 q = mul2(pj, inv2);
-            const float2 df = sub2(q, sub2(add2(q, magic2), magic2));
-            if (fmaxf(fabsf(df.x), fabsf(df.y)) > tie_lim) {
-              const float2 rq = make_float2(round_magic(__fdiv_rn(pj.x, step)), round_magic(__fdiv_rn(pj.y, step)));
-              const float2 d = sub2(w[j], mul2(mul2(rq, step2), rsv[j]));
-              outw[j] = pack_bf16x2(d.x, d.y);
-            }
-          }
-        }
-      }
-      uint4* dst = reinterpret_cast<uint4*>(dW + ((int64_t)k * C2 + row) * C1 + c0);
-      if (!fast) {
-        if (col_ok)
-          delta16_general(&tile[r][lane * 2], s_tab + (int64_t)k * C1 + c0, rs_tab + (int64_t)k * C1 + c0, mn, step, inv,
-                          qmax_f, dst);
-      } else if (col_ok) {
-        dst[0] = make_uint4(outw[0], outw[1], outw[2], outw[3]);
-        dst[1] = make_uint4(outw[4], outw[5], outw[6], outw[7]);
-      }
+      if (row0 + r >= C2) break;                  // rows of a warp ascend with p; shuffles below stay warp-uniform
+      RowHead h;
+      row_head(tile[r][lane * 2], tile[r][lane * 2 + 1], sv, lanes_per_group, qmax_f, tie_lim, h);
+      row_tail(h, sv, rsv, tie_lim, qmax_f, col_ok, &tile[r][lane * 2], s_tab + (int64_t)k * C1 + c0,
+               rs_tab + (int64_t)k * C1 + c0, reinterpret_cast<uint4*>(dW + ((int64_t)k * C2 + row0 + r) * C1 + c0));
     }
   }
 }
@@ -436,8 +461,9 @@ int launch_fakequant_group(const uint16_t* W, const uint16_t* s, const float* rs
 // max|value| / qpos, code = rint(value / step) (Sec. 2.2, first two equations; qpos = 2^(n-1) - 1).
 //
 // A row's maximum couples all of its channels, so the work is split in two fully parallel passes
-// over the same 32-row x 512-channel tiles as the group kernels, each tile staged once in shared
-// memory and re-used for every candidate:
+// over 512-channel tiles (32 rows in pass 1, 16 in pass 2).  A thread owns 16 channels of its rows and keeps them, unpacked
+// to binary32 pairs, in registers for all of its candidates (read straight from global memory: a warp
+// covers 1 KB of a row), so a candidate costs it one load of the 16 multipliers and the arithmetic:
 //   pass 1  per (candidate, row) the maximum |value| over the tile's channels -> atomic max on the
 //           float's bit pattern (non-negative floats order like integers, so the result does not
 //           depend on arrival order); a one-line kernel then turns the maxima into steps in place;
@@ -449,105 +475,103 @@ int launch_fakequant_group(const uint16_t* W, const uint16_t* s, const float* rs
 // binary32 reciprocal for activations (from the table, or taken here from a bf16 scale), or 1.
 // ------------------------------------------------------------------------------------------------
 enum MultKind { kMultScale = 0, kMultRecipTable = 1, kMultRecipOfScale = 2 };
+constexpr int kAmaxRowsPerThread = 4;      // pass 1: 32-row tiles (the multipliers of a candidate serve four rows)
+constexpr int kCodeRowsPerThread = 2;      // pass 2: 16-row tiles (its temporaries leave room for two rows)
 
 template <int kKind>
-__device__ __forceinline__ void load_mult16(const uint16_t* s_row, const float* rs_row, int64_t c0, bool col_ok,
-                                            float2 (&m)[8]) {
+__device__ __forceinline__ void load_mult_pairs(const uint16_t* s_row, const float* rs_row, int64_t c0, bool col_ok,
+                                                f32x2 (&m)[8]) {
   if (!col_ok || (kKind != kMultRecipTable && s_row == nullptr)) {
 #pragma unroll
-    for (int j = 0; j < 8; ++j) m[j] = make_float2(1.0f, 1.0f);
+    for (int j = 0; j < 8; ++j) m[j] = pair_of(1.0f, 1.0f);
     return;
   }
   if (kKind == kMultRecipTable) {
-    const float4* rp = reinterpret_cast<const float4*>(rs_row + c0);
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const float4 r4 = rp[j];
-      m[2 * j] = make_float2(r4.x, r4.y);
-      m[2 * j + 1] = make_float2(r4.z, r4.w);
-    }
+    load_pairs16(rs_row + c0, m);
   } else {
     const uint4* sp = reinterpret_cast<const uint4*>(s_row + c0);
-    const uint4 a = sp[0], b = sp[1];
-    m[0] = unpack2(a.x); m[1] = unpack2(a.y); m[2] = unpack2(a.z); m[3] = unpack2(a.w);
-    m[4] = unpack2(b.x); m[5] = unpack2(b.y); m[6] = unpack2(b.z); m[7] = unpack2(b.w);
+    unpack16_pairs(sp[0], sp[1], m);
     if (kKind == kMultRecipOfScale) {
 #pragma unroll
-      for (int j = 0; j < 8; ++j) m[j] = make_float2(__fdiv_rn(1.0f, m[j].x), __fdiv_rn(1.0f, m[j].y));
+      for (int j = 0; j < 8; ++j) {
+        const float2 v = halves(m[j]);
+        m[j] = pair_of(__fdiv_rn(1.0f, v.x), __fdiv_rn(1.0f, v.y));
+      }
     }
   }
 }
 
-__device__ __forceinline__ void stage_tile(uint4 (*tile)[kGqCols / 8], const uint16_t* __restrict__ src, int64_t row0,
-                                           int64_t R, int64_t C1, int64_t c0, bool col_ok, int warp, int lane) {
+// This thread's 16 channels of its rows (rows warp, warp + 8, ... of the tile), zeros outside the matrix.
+template <int kRows>
+__device__ __forceinline__ void load_rows_to_registers(const uint16_t* __restrict__ src, int64_t row0, int64_t R,
+                                                       int64_t C1, int64_t c0, bool col_ok, int warp,
+                                                       f32x2 (&w)[kRows][8]) {
+  uint4 raw[kRows][2];
 #pragma unroll
-  for (int p = 0; p < kRowRows / 8; ++p) {
-    const int r = p * 8 + warp;
-    uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0;
-    if (col_ok && row0 + r < R) {
-      const uint16_t* sp = src + (row0 + r) * C1 + c0;
-      v0 = ld_nc_16(sp);
-      v1 = ld_nc_16(sp + 8);
+  for (int p = 0; p < kRows; ++p) {            // all loads first, then the unpacking
+    const int64_t row = row0 + p * 8 + warp;
+    raw[p][0] = raw[p][1] = make_uint4(0, 0, 0, 0);
+    if (col_ok && row < R) {
+      const uint16_t* sp = src + row * C1 + c0;
+      raw[p][0] = ld_nc_16(sp);
+      raw[p][1] = ld_nc_16(sp + 8);
     }
-    tile[r][lane * 2] = v0;
-    tile[r][lane * 2 + 1] = v1;
   }
-  __syncthreads();
-}
-
-__device__ __forceinline__ void unpack16(const uint4& t0, const uint4& t1, float2 (&w)[8]) {
-  w[0] = unpack2(t0.x); w[1] = unpack2(t0.y); w[2] = unpack2(t0.z); w[3] = unpack2(t0.w);
-  w[4] = unpack2(t1.x); w[5] = unpack2(t1.y); w[6] = unpack2(t1.z); w[7] = unpack2(t1.w);
+#pragma unroll
+  for (int p = 0; p < kRows; ++p) unpack16_pairs(raw[p][0], raw[p][1], w[p]);
 }
 
 template <int kKind>
-__global__ void __launch_bounds__(kGqThreads, 3)
+__global__ void __launch_bounds__(kGqThreads, 2)
 row_amax_kernel(const uint16_t* __restrict__ src, const uint16_t* __restrict__ s_tab, const float* __restrict__ rs_tab,
                 int K, int k_per_cta, int64_t R_all, const int32_t* __restrict__ n_rows_dev, int64_t C1,
                 int* __restrict__ amax_bits /*[K,R_all], zeroed*/) {
-  extern __shared__ uint4 tile_dyn[];
-  uint4 (*tile)[kGqCols / 8] = reinterpret_cast<uint4 (*)[kGqCols / 8]>(tile_dyn);
+  constexpr int kRows = kAmaxRowsPerThread;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t col_blocks = (C1 + kGqCols - 1) / kGqCols;      // grid.x = column blocks x row tiles, columns fastest
   const int64_t c0 = (int64_t)(blockIdx.x % col_blocks) * kGqCols + lane * 16;
-  const int64_t row0 = (int64_t)(blockIdx.x / col_blocks) * kRowRows;
+  const int64_t row0 = (int64_t)(blockIdx.x / col_blocks) * (kRows * 8);
   const int64_t R = (n_rows_dev != nullptr) ? (int64_t)*n_rows_dev : R_all;    // rows beyond are not live
   if (row0 >= R) return;                                                        // the whole CTA leaves together
   const bool col_ok = c0 < C1;
-  stage_tile(tile, src, row0, R, C1, c0, col_ok, warp, lane);
+  f32x2 w[kRows][8];
+  load_rows_to_registers<kRows>(src, row0, R, C1, c0, col_ok, warp, w);
   const int k_begin = blockIdx.y * k_per_cta;
   const int k_end = min(K, k_begin + k_per_cta);
-  for (int k = k_begin; k < k_end; ++k) {
-    float2 m[8];
-    load_mult16<kKind>(s_tab ? s_tab + (int64_t)k * C1 : nullptr, rs_tab ? rs_tab + (int64_t)k * C1 : nullptr, c0,
-                       col_ok, m);
-    // four of the warp's rows at a time: four independent shuffle chains instead of one after the other
-#pragma unroll 1
-    for (int h = 0; h < kRowRows / 32; ++h) {
-      float a[4];
+  auto mult_of = [&](int k, f32x2 (&m)[8]) {
+    load_mult_pairs<kKind>(s_tab ? s_tab + (int64_t)k * C1 : nullptr, rs_tab ? rs_tab + (int64_t)k * C1 : nullptr, c0,
+                           col_ok, m);
+  };
+  // one candidate: the next candidate's multipliers are requested before this one's arithmetic starts
+  auto candidate = [&](int k, const f32x2 (&m)[8], f32x2 (&m_next)[8]) {
+    if (k + 1 < k_end) mult_of(k + 1, m_next);
+    float a[kRows];
 #pragma unroll
-      for (int p = 0; p < 4; ++p) {
-        const int r = (h * 4 + p) * 8 + warp;          // rows past the end were staged as zeros
-        float2 w[8];
-        unpack16(tile[r][lane * 2], tile[r][lane * 2 + 1], w);
-        a[p] = 0.0f;
+    for (int p = 0; p < kRows; ++p) {
+      a[p] = 0.0f;                                    // rows and channels outside the matrix were loaded as zeros
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const float2 v = mul2(w[j], m[j]);
-          a[p] = max3(a[p], fabsf(v.x), fabsf(v.y));
-        }
+      for (int j = 0; j < 8; ++j) {
+        const float2 v = halves(pmul(w[p][j], m[j]));
+        a[p] = max3(a[p], fabsf(v.x), fabsf(v.y));
       }
-#pragma unroll
-      for (int off = 16; off > 0; off >>= 1) {
-#pragma unroll
-        for (int p = 0; p < 4; ++p) a[p] = fmaxf(a[p], __shfl_xor_sync(0xFFFFFFFFu, a[p], off));
-      }
-      float mine = a[0];
-#pragma unroll
-      for (int p = 1; p < 4; ++p) mine = (lane == p) ? a[p] : mine;
-      const int64_t my_row = row0 + (h * 4 + lane) * 8 + warp;
-      if (lane < 4 && my_row < R) atomicMax(amax_bits + (int64_t)k * R_all + my_row, __float_as_int(mine));
     }
+    // independent shuffle chains, one per row, instead of one after the other
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+#pragma unroll
+      for (int p = 0; p < kRows; ++p) a[p] = fmaxf(a[p], __shfl_xor_sync(0xFFFFFFFFu, a[p], off));
+    }
+    float mine = a[0];
+#pragma unroll
+    for (int p = 1; p < kRows; ++p) mine = (lane == p) ? a[p] : mine;
+    const int64_t my_row = row0 + lane * 8 + warp;
+    if (lane < kRows && my_row < R) atomicMax(amax_bits + (int64_t)k * R_all + my_row, __float_as_int(mine));
+  };
+  f32x2 ma[8], mb[8];
+  mult_of(k_begin, ma);
+  for (int k = k_begin; k < k_end; k += 2) {
+    candidate(k, ma, mb);
+    if (k + 1 < k_end) candidate(k + 1, mb, ma);
   }
 }
 
@@ -557,331 +581,128 @@ __global__ void amax_to_step_kernel(float* __restrict__ v, int64_t n, float qpos
 }
 
 // One thread's 16 codes with the exact division (a near-tie was seen on the straight-line path).
-__device__ __noinline__ void codes16_exact(const uint4* tile16, const float* mult16, float st, float qpos, uint4* dst) {
+struct Pairs8 {
+  f32x2 v[8];
+};
+__device__ __noinline__ void codes16_exact(Pairs8 w, Pairs8 m, float st, float qpos, uint4* dst) {
   uint32_t pk[4] = {0u, 0u, 0u, 0u};
-#pragma unroll 1
-  for (int h = 0; h < 2; ++h) {
-    float w[8];
-    unpack8(tile16[h], w);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const float v = __fmul_rn(w[j], mult16[h * 8 + j]);
-      const float q = fminf(fmaxf(__fdiv_rn(v, st), -qpos - 1.0f), qpos);
-      const int e = h * 8 + j;
-      pk[e >> 2] |= (__float_as_uint(__fadd_rn(q, kMagic)) & 0xFFu) << ((e & 3) * 8);
-    }
+  for (int j = 0; j < 8; ++j) {
+    const float2 wv = halves(w.v[j]), mv = halves(m.v[j]);
+    const float q0 = fminf(fmaxf(__fdiv_rn(__fmul_rn(wv.x, mv.x), st), -qpos - 1.0f), qpos);
+    const float q1 = fminf(fmaxf(__fdiv_rn(__fmul_rn(wv.y, mv.y), st), -qpos - 1.0f), qpos);
+    const int e = 2 * j;
+    pk[e >> 2] |= (__float_as_uint(__fadd_rn(q0, kMagic)) & 0xFFu) << ((e & 3) * 8);
+    pk[e >> 2] |= (__float_as_uint(__fadd_rn(q1, kMagic)) & 0xFFu) << (((e + 1) & 3) * 8);
   }
   *dst = make_uint4(pk[0], pk[1], pk[2], pk[3]);
 }
 
 template <int kKind>
-__global__ void __launch_bounds__(kGqThreads, 3)
+__global__ void __launch_bounds__(kGqThreads, 2)
 row_codes_kernel(const uint16_t* __restrict__ src, const uint16_t* __restrict__ s_tab, const float* __restrict__ rs_tab,
                  const float* __restrict__ step /*[K,R_all]*/, int K, int k_per_cta, int64_t R_all,
                  const int32_t* __restrict__ n_rows_dev, int64_t C1, float qpos, float tie_eps,
                  int8_t* __restrict__ q /*[K,R_all,C1]*/) {
-  extern __shared__ uint4 tile_dyn[];
-  uint4 (*tile)[kGqCols / 8] = reinterpret_cast<uint4 (*)[kGqCols / 8]>(tile_dyn);
+  constexpr int kRows = kCodeRowsPerThread;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t col_blocks = (C1 + kGqCols - 1) / kGqCols;      // grid.x = column blocks x row tiles, columns fastest
   const int64_t c0 = (int64_t)(blockIdx.x % col_blocks) * kGqCols + lane * 16;
-  const int64_t row0 = (int64_t)(blockIdx.x / col_blocks) * kRowRows;
+  const int64_t row0 = (int64_t)(blockIdx.x / col_blocks) * (kRows * 8);
   const int64_t R = (n_rows_dev != nullptr) ? (int64_t)*n_rows_dev : R_all;
-  if (row0 >= R) return;
-  const bool col_ok = c0 < C1;
-  stage_tile(tile, src, row0, R, C1, c0, col_ok, warp, lane);
-  if (!col_ok) return;                    // no warp-wide operation below
+  if (row0 >= R || c0 >= C1) return;      // no warp-wide operation below
+  f32x2 w[kRows][8];
+  load_rows_to_registers<kRows>(src, row0, R, C1, c0, true, warp, w);
   const float tie_lim = 0.5f - tie_eps;
-  const float2 magic2 = make_float2(kMagic, kMagic);
+  const f32x2 magic2 = pair_of(kMagic, kMagic);
   const int k_begin = blockIdx.y * k_per_cta;
   const int k_end = min(K, k_begin + k_per_cta);
-  for (int k = k_begin; k < k_end; ++k) {
-    float2 m[8];
-    load_mult16<kKind>(s_tab ? s_tab + (int64_t)k * C1 : nullptr, rs_tab ? rs_tab + (int64_t)k * C1 : nullptr, c0,
-                       true, m);
-#pragma unroll 1
-    for (int p = 0; p < kRowRows / 8; ++p) {
-      const int r = p * 8 + warp;
-      const int64_t row = row0 + r;
-      if (row >= R) break;
-      const float st = step[(int64_t)k * R_all + row];
-      const float inv = rcp_fast(st);
-      const float2 inv2 = make_float2(inv, inv);
-      float2 w[8];
-      unpack16(tile[r][lane * 2], tile[r][lane * 2 + 1], w);
-      float near = 0.0f;
-      uint32_t tb[16];
+  // what a candidate needs from memory: its 16 multipliers and the steps of this thread's rows
+  auto fetch = [&](int k, f32x2 (&m)[8], float (&st)[kRows]) {
+    load_mult_pairs<kKind>(s_tab ? s_tab + (int64_t)k * C1 : nullptr, rs_tab ? rs_tab + (int64_t)k * C1 : nullptr, c0,
+                           true, m);
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const float2 qv = mul2(mul2(w[j], m[j]), inv2);
-        const float2 t = add2(qv, magic2);           // low mantissa byte = the code in two's complement
-        const float2 df = sub2(qv, sub2(t, magic2));
-        near = max3(near, fabsf(df.x), fabsf(df.y));
-        tb[2 * j] = __float_as_uint(t.x);
-        tb[2 * j + 1] = __float_as_uint(t.y);
-      }
-      uint4* dst = reinterpret_cast<uint4*>(q + ((int64_t)k * R_all + row) * C1 + c0);
-      if (near > tie_lim) {
-        float mf[16];
+    for (int p = 0; p < kRows; ++p) {
+      const int64_t row = row0 + p * 8 + warp;
+      st[p] = row < R ? step[(int64_t)k * R_all + row] : 1.0f;
+    }
+  };
+  // one candidate: the next candidate's operands are requested before this one's arithmetic starts
+  auto candidate = [&](int k, const f32x2 (&m)[8], const float (&st)[kRows], f32x2 (&m_next)[8], float (&st_next)[kRows]) {
+    if (k + 1 < k_end) fetch(k + 1, m_next, st_next);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { mf[2 * j] = m[j].x; mf[2 * j + 1] = m[j].y; }
-        codes16_exact(&tile[r][lane * 2], mf, st, qpos, dst);
-      } else {
-        uint32_t pk[4];
+    for (int p = 0; p < kRows; ++p) {
+      const int64_t row = row0 + p * 8 + warp;
+      if (row < R) {
+        const float inv = rcp_fast(st[p]);
+        const f32x2 inv2 = pair_of(inv, inv);
+        float near = 0.0f;
+        uint32_t tb[16];
 #pragma unroll
-        for (int g = 0; g < 4; ++g)
-          pk[g] = __byte_perm(__byte_perm(tb[4 * g], tb[4 * g + 1], 0x0040), __byte_perm(tb[4 * g + 2], tb[4 * g + 3], 0x0040),
-                              0x5410);
-        *dst = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        for (int j = 0; j < 8; ++j) {
+          const f32x2 qv = pmul(pmul(w[p][j], m[j]), inv2);
+          const f32x2 t = padd(qv, magic2);             // low mantissa byte = the code in two's complement
+          const float2 df = halves(psub(qv, psub(t, magic2)));
+          near = max3(near, fabsf(df.x), fabsf(df.y));
+          const float2 th = halves(t);
+          tb[2 * j] = __float_as_uint(th.x);
+          tb[2 * j + 1] = __float_as_uint(th.y);
+        }
+        uint4* dst = reinterpret_cast<uint4*>(q + ((int64_t)k * R_all + row) * C1 + c0);
+        if (near > tie_lim) {
+          Pairs8 wp, mp;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) { wp.v[j] = w[p][j]; mp.v[j] = m[j]; }
+          codes16_exact(wp, mp, st[p], qpos, dst);
+        } else {
+          uint32_t pk[4];
+#pragma unroll
+          for (int g = 0; g < 4; ++g)
+            pk[g] = __byte_perm(__byte_perm(tb[4 * g], tb[4 * g + 1], 0x0040), __byte_perm(tb[4 * g + 2], tb[4 * g + 3], 0x0040),
+                                0x5410);
+          *dst = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
       }
     }
+  };
+  f32x2 ma[8], mb[8];
+  float sta[kRows], stb[kRows];
+  fetch(k_begin, ma, sta);
+  for (int k = k_begin; k < k_end; k += 2) {
+    candidate(k, ma, sta, mb, stb);
+    if (k + 1 < k_end) candidate(k + 1, mb, stb, ma, sta);
   }
 }
 
 template <int kKind>
-static int launch_rows_two_pass(const uint16_t* src, const uint16_t* s, const float* rs, int K, int64_t R, int64_t C1, int bits,
+static int launch_rows(const uint16_t* src, const uint16_t* s, const float* rs, int K, int64_t R, int64_t C1, int bits,
                        int8_t* q, float* step, const int32_t* n_rows_dev, cudaStream_t st) {
-  static OncePerDevice once;      // one per instantiation of this template
-  int rc = once_per_device(once, [] {
-    const cudaError_t e = cudaFuncSetAttribute(row_amax_kernel<kKind>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kRowSmem);
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(row_codes_kernel<kKind>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kRowSmem);
-  });
-  if (rc != TLQ_OK) return rc;
   const int sms = device_sm_count();
   if (sms <= 0) return TLQ_ERR_CUDA;
-  const int64_t ctas = ceil_div(C1, kGqCols) * ceil_div(R, kRowRows);
-  int64_t kchunks = ceil_div((int64_t)sms * 6, ctas);
-  if (kchunks > K) kchunks = K;
-  if (kchunks < 1) kchunks = 1;
-  const int k_per_cta = (int)ceil_div(K, kchunks);
-  kchunks = ceil_div(K, k_per_cta);
-  const dim3 grid((unsigned)(ceil_div(C1, kGqCols) * ceil_div(R, kRowRows)), (unsigned)kchunks);
+  // candidates are split over grid.y only when the tiles alone would not fill the machine several times over
+  auto shape = [&](int tile_rows, int& k_per_cta) {
+    const int64_t tiles = ceil_div(C1, kGqCols) * ceil_div(R, tile_rows);
+    int64_t kchunks = ceil_div((int64_t)sms * 6, tiles);
+    if (kchunks > K) kchunks = K;
+    if (kchunks < 1) kchunks = 1;
+    k_per_cta = (int)ceil_div(K, kchunks);
+    return dim3((unsigned)tiles, (unsigned)ceil_div(K, k_per_cta));
+  };
+  int kpc_amax = 1, kpc_codes = 1;
+  const dim3 grid_amax = shape(kAmaxRowsPerThread * 8, kpc_amax);
+  const dim3 grid_codes = shape(kCodeRowsPerThread * 8, kpc_codes);
   const float qpos = (float)((1 << (bits - 1)) - 1);
   const float tie_eps = 4.0e-7f * (qpos + 1.0f);
   const int64_t n = (int64_t)K * R;
   TLQ_CUDA_TRY(cudaMemsetAsync(step, 0, (size_t)n * sizeof(float), st));
-  row_amax_kernel<kKind><<<grid, kGqThreads, kRowSmem, st>>>(src, s, rs, K, k_per_cta, R, n_rows_dev, C1,
-                                                      reinterpret_cast<int*>(step));
-  rc = after_launch();
+  row_amax_kernel<kKind><<<grid_amax, kGqThreads, 0, st>>>(src, s, rs, K, kpc_amax, R, n_rows_dev, C1,
+                                                     reinterpret_cast<int*>(step));
+  int rc = after_launch();
   if (rc != TLQ_OK) return rc;
   amax_to_step_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(step, n, qpos);
   if ((rc = after_launch()) != TLQ_OK) return rc;
-  row_codes_kernel<kKind><<<grid, kGqThreads, kRowSmem, st>>>(src, s, rs, step, K, k_per_cta, R, n_rows_dev, C1, qpos, tie_eps, q);
+  row_codes_kernel<kKind><<<grid_codes, kGqThreads, 0, st>>>(src, s, rs, step, K, kpc_codes, R, n_rows_dev, C1, qpos, tie_eps, q);
   return after_launch();
-}
-
-// ------------------------------------------------------------------------------------------------
-// The same quantizer with whole rows resident in one CTA: one launch instead of four, the source read
-// from HBM once, and per element about half the instructions of the two tiled passes above.
-//
-// A CTA stages RB complete rows in shared memory (RB x C1 bf16, at most ~100 KB so that two CTAs share
-// an SM) and walks its candidates in order.  A thread owns fixed 16-channel columns, so the candidate's
-// per-channel multipliers are loaded once per column and serve all RB rows.  While the codes of
-// candidate k are formed, the same unpacked values are multiplied by candidate k+1's multipliers and
-// folded into running row maxima; the maxima are combined across the CTA (shuffles, then one warp per
-// row), which yields step and 1/step of candidate k+1 for the next round.  Only the first candidate of
-// a CTA needs a maximum pass of its own.  Per (row, candidate) the result is what the tiled passes
-// give: max over channels of |value| is taken over the same binary32 products, the step is the same
-// IEEE division, the codes come from the same straight-line arithmetic with the exact-division fix-up.
-// ------------------------------------------------------------------------------------------------
-constexpr int kFusedThreads = 256;
-constexpr int kFusedWarps = kFusedThreads / 32;
-constexpr size_t kFusedSmemBudget = 100 << 10;     // two CTAs per SM
-constexpr size_t kFusedSmemLimit = 220 << 10;      // one CTA per SM: the widest row this kernel takes
-
-template <int kKind, int RB>
-__global__ void __launch_bounds__(kFusedThreads, 2)
-row_quant_fused_kernel(const uint16_t* __restrict__ src, const uint16_t* __restrict__ s_tab,
-                       const float* __restrict__ rs_tab, int K, int k_per_cta, int64_t R_all,
-                       const int32_t* __restrict__ n_rows_dev, int64_t C1, float qpos, float tie_eps,
-                       int8_t* __restrict__ q /*[K,R_all,C1]*/, float* __restrict__ step /*[K,R_all]*/) {
-  extern __shared__ uint4 tile_dyn[];                 // [RB][C1 / 8]
-  __shared__ float red[2][kFusedWarps][RB];           // per-warp row maxima of the candidate being prepared
-  __shared__ float2 step_inv[2][RB];                  // (step, ~1/step) per row, double-buffered over candidates
-  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
-  const int64_t R = (n_rows_dev != nullptr) ? (int64_t)*n_rows_dev : R_all;    // rows beyond are not live
-  const int64_t row0 = (int64_t)blockIdx.x * RB;
-  if (row0 >= R) return;                              // the whole CTA leaves together
-  const int nchunks = (int)(C1 >> 4);                 // 16-channel columns of a row
-  const int row_u4 = nchunks * 2;                     // uint4 per staged row
-  const int k_begin = blockIdx.y * k_per_cta;
-  const int k_end = min(K, k_begin + k_per_cta);
-
-  for (int i = t; i < RB * row_u4; i += kFusedThreads) {
-    const int r = i / row_u4, c = i - r * row_u4;
-    uint4 v = make_uint4(0, 0, 0, 0);                 // rows past the end count as zeros and store nothing
-    if (row0 + r < R) v = ld_nc_16(src + (row0 + r) * C1 + (int64_t)c * 8);
-    tile_dyn[i] = v;
-  }
-  // Narrow rows leave threads over: they are dealt out over row groups, thread (rg, column) taking rows rg, rg + groups, ...
-  const int col_threads = nchunks < kFusedThreads ? nchunks : kFusedThreads;
-  const int groups = kFusedThreads / col_threads;
-  const int rg = t / col_threads;
-  const int col0 = t - rg * col_threads;
-  uint32_t row_mask = 0;
-  if (rg < groups)
-    for (int r = rg; r < RB; r += groups) row_mask |= 1u << r;
-  __syncthreads();
-
-  const float tie_lim = 0.5f - tie_eps;
-  const float2 magic2 = make_float2(kMagic, kMagic);
-  auto mult_rows = [&](int k, const uint16_t*& s_row, const float*& rs_row) {
-    s_row = s_tab ? s_tab + (int64_t)k * C1 : nullptr;
-    rs_row = rs_tab ? rs_tab + (int64_t)k * C1 : nullptr;
-  };
-  // Combine the threads' running maxima of candidate k into (step, 1/step) per row; buffer `par`.
-  auto publish = [&](float (&am)[RB], int par, int k) {
-#pragma unroll
-    for (int r = 0; r < RB; ++r) {
-      float v = am[r];
-#pragma unroll
-      for (int off = 16; off > 0; off >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, off));
-      if (lane == 0) red[par][warp][r] = v;
-    }
-    __syncthreads();
-    if (warp < RB) {                                  // warp w finishes row w
-      float v = lane < kFusedWarps ? red[par][lane][warp] : 0.0f;
-#pragma unroll
-      for (int off = kFusedWarps / 2; off > 0; off >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, off));
-      if (lane == 0) {
-        const float st = __fdiv_rn(fmaxf(v, TLQ_RANGE_FLOOR), qpos);
-        step_inv[par][warp] = make_float2(st, rcp_fast(st));
-        if (row0 + warp < R) step[(int64_t)k * R_all + row0 + warp] = st;
-      }
-    }
-    __syncthreads();
-  };
-
-  float am[RB];
-#pragma unroll
-  for (int r = 0; r < RB; ++r) am[r] = 0.0f;
-  if (row_mask != 0) {                                // the first candidate's maxima: a pass of its own
-    const uint16_t* s_row; const float* rs_row;
-    mult_rows(k_begin, s_row, rs_row);
-    for (int ch = col0; ch < nchunks; ch += col_threads) {
-      float2 m[8];
-      load_mult16<kKind>(s_row, rs_row, (int64_t)ch * 16, true, m);
-#pragma unroll
-      for (int r = 0; r < RB; ++r) {
-        if (!((row_mask >> r) & 1u)) continue;
-        float2 w[8];
-        unpack16(tile_dyn[r * row_u4 + ch * 2], tile_dyn[r * row_u4 + ch * 2 + 1], w);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const float2 v = mul2(w[j], m[j]);
-          am[r] = max3(am[r], fabsf(v.x), fabsf(v.y));
-        }
-      }
-    }
-  }
-  publish(am, 0, k_begin);
-
-  for (int k = k_begin; k < k_end; ++k) {
-    const int par = (k - k_begin) & 1;
-    const bool has_next = k + 1 < k_end;
-    float st[RB], inv[RB];
-#pragma unroll
-    for (int r = 0; r < RB; ++r) {
-      const float2 si = step_inv[par][r];
-      st[r] = si.x; inv[r] = si.y;
-      am[r] = 0.0f;
-    }
-    if (row_mask != 0) {
-      const uint16_t* s_row; const float* rs_row;
-      const uint16_t* s_next = nullptr; const float* rs_next = nullptr;
-      mult_rows(k, s_row, rs_row);
-      if (has_next) mult_rows(k + 1, s_next, rs_next);
-      for (int ch = col0; ch < nchunks; ch += col_threads) {
-        float2 m[8], m2[8];
-        load_mult16<kKind>(s_row, rs_row, (int64_t)ch * 16, true, m);
-        if (has_next) load_mult16<kKind>(s_next, rs_next, (int64_t)ch * 16, true, m2);
-#pragma unroll
-        for (int r = 0; r < RB; ++r) {
-          if (!((row_mask >> r) & 1u)) continue;
-          const uint4* tile16 = &tile_dyn[r * row_u4 + ch * 2];
-          float2 w[8];
-          unpack16(tile16[0], tile16[1], w);
-          if (has_next) {
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              const float2 v = mul2(w[j], m2[j]);
-              am[r] = max3(am[r], fabsf(v.x), fabsf(v.y));
-            }
-          }
-          const int64_t row = row0 + r;
-          if (row >= R) continue;
-          const float2 inv2 = make_float2(inv[r], inv[r]);
-          float near = 0.0f;
-          uint32_t tb[16];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const float2 qv = mul2(mul2(w[j], m[j]), inv2);
-            const float2 tt = add2(qv, magic2);          // low mantissa byte = the code in two's complement
-            const float2 df = sub2(qv, sub2(tt, magic2));
-            near = max3(near, fabsf(df.x), fabsf(df.y));
-            tb[2 * j] = __float_as_uint(tt.x);
-            tb[2 * j + 1] = __float_as_uint(tt.y);
-          }
-          uint4* dst = reinterpret_cast<uint4*>(q + ((int64_t)k * R_all + row) * C1 + (int64_t)ch * 16);
-          if (near > tie_lim) {
-            float mf[16];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) { mf[2 * j] = m[j].x; mf[2 * j + 1] = m[j].y; }
-            codes16_exact(tile16, mf, st[r], qpos, dst);
-          } else {
-            uint32_t pk[4];
-#pragma unroll
-            for (int g = 0; g < 4; ++g)
-              pk[g] = __byte_perm(__byte_perm(tb[4 * g], tb[4 * g + 1], 0x0040),
-                                  __byte_perm(tb[4 * g + 2], tb[4 * g + 3], 0x0040), 0x5410);
-            *dst = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-          }
-        }
-      }
-    }
-    if (has_next) publish(am, par ^ 1, k + 1);
-  }
-}
-
-template <int kKind, int RB>
-static int launch_rows_fused(const uint16_t* src, const uint16_t* s, const float* rs, int K, int64_t R, int64_t C1,
-                             int bits, int8_t* q, float* step, const int32_t* n_rows_dev, cudaStream_t st) {
-  static OncePerDevice once;
-  int rc = once_per_device(once, [] {
-    return cudaFuncSetAttribute(row_quant_fused_kernel<kKind, RB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)kFusedSmemLimit);
-  });
-  if (rc != TLQ_OK) return rc;
-  const int sms = device_sm_count();
-  if (sms <= 0) return TLQ_ERR_CUDA;
-  const int64_t row_blocks = ceil_div(R, RB);
-  int64_t kchunks = ceil_div((int64_t)sms * 12, row_blocks);     // several work units per resident CTA
-  if (kchunks > K) kchunks = K;
-  if (kchunks < 1) kchunks = 1;
-  const int k_per_cta = (int)ceil_div(K, kchunks);
-  kchunks = ceil_div(K, k_per_cta);
-  const dim3 grid((unsigned)row_blocks, (unsigned)kchunks);
-  const float qpos = (float)((1 << (bits - 1)) - 1);
-  const float tie_eps = 4.0e-7f * (qpos + 1.0f);
-  const size_t smem = (size_t)RB * (size_t)C1 * 2;
-  row_quant_fused_kernel<kKind, RB><<<grid, kFusedThreads, smem, st>>>(src, s, rs, K, k_per_cta, R, n_rows_dev, C1, qpos,
-                                                                  tie_eps, q, step);
-  return after_launch();
-}
-
-// Rows per CTA of the whole-row kernel: the largest of 8, 4, 2, 1 whose rows fit the shared-memory budget; rows too
-// wide even for one per CTA go through the two tiled passes.
-template <int kKind>
-static int launch_rows(const uint16_t* src, const uint16_t* s, const float* rs, int K, int64_t R, int64_t C1, int bits,
-                       int8_t* q, float* step, const int32_t* n_rows_dev, cudaStream_t st) {
-  const size_t row_bytes = (size_t)C1 * 2;
-  if ((C1 & 15) != 0 || row_bytes > kFusedSmemLimit)
-    return launch_rows_two_pass<kKind>(src, s, rs, K, R, C1, bits, q, step, n_rows_dev, st);
-  if (8 * row_bytes <= kFusedSmemBudget) return launch_rows_fused<kKind, 8>(src, s, rs, K, R, C1, bits, q, step, n_rows_dev, st);
-  if (4 * row_bytes <= kFusedSmemBudget) return launch_rows_fused<kKind, 4>(src, s, rs, K, R, C1, bits, q, step, n_rows_dev, st);
-  if (2 * row_bytes <= kFusedSmemBudget) return launch_rows_fused<kKind, 2>(src, s, rs, K, R, C1, bits, q, step, n_rows_dev, st);
-  return launch_rows_fused<kKind, 1>(src, s, rs, K, R, C1, bits, q, step, n_rows_dev, st);
 }
 
 int launch_fakequant_rows_i8(const uint16_t* W, const uint16_t* s, int K, int64_t C2, int64_t C1, int bits, int8_t* q,

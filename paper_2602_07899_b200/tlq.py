@@ -31,7 +31,7 @@ EXPORTS = (
     "tlq_status_string", "tlq_version", "tlq_token_importance", "tlq_scale_candidates_workspace_bytes",
     "tlq_scale_candidates", "tlq_scale_candidates_noalloc", "tlq_quantize_weights", "tlq_pack_codes4", "tlq_quantize_activations", "tlq_scale_search_workspace_bytes", "tlq_scale_search_layer", "tlq_scale_search_layer_two_stream",
     "tlq_apply_layer_workspace_bytes", "tlq_apply_layer", "tlq_read_status", "tlq_stage_timing_enable",
-    "tlq_stage_timing_drain", "tlq_kernel_launch_count",
+    "tlq_stage_timing_drain", "tlq_kernel_launch_count", "tlq_selftest_bounded_wait",
 )
 
 
@@ -92,6 +92,8 @@ def _load() -> ctypes.CDLL:
     lib.tlq_apply_layer_workspace_bytes.argtypes = [i64, i64, i64, cfgp]
     lib.tlq_apply_layer.argtypes = [vp, i64, i64, vp, i64, vp, vp, cfgp, vp, sz, vp, vp, vp, vp, vp]
     lib.tlq_read_status.argtypes = [vp, vp]
+    lib.tlq_selftest_bounded_wait.argtypes = [vp, sz, i64, vp]
+    lib.tlq_selftest_bounded_wait.restype = i32
     lib.tlq_stage_timing_enable.argtypes = [i32]
     lib.tlq_stage_timing_drain.argtypes = [ctypes.POINTER(ctypes.c_float), i32]
     for fn in ("tlq_token_importance", "tlq_scale_candidates", "tlq_scale_candidates_noalloc", "tlq_quantize_weights", "tlq_pack_codes4", "tlq_quantize_activations", "tlq_scale_search_layer",
@@ -281,6 +283,15 @@ def tlq_apply_layer(X: torch.Tensor, W: torch.Tensor, s: Optional[torch.Tensor],
 
 def tlq_read_status(workspace: torch.Tensor, stream=None) -> int:
     return int(lib.tlq_read_status(_ptr(workspace), _stream(stream)))
+
+
+def tlq_selftest_bounded_wait(workspace: torch.Tensor, limit_cycles: int = 2_000_000, stream=None) -> int:
+    """Run the bounded-wait self-test on `workspace` and return the device status it left (TLQ_ERR_TIMEOUT when
+    the error path works).  Synchronises the stream."""
+    st = _stream(stream)
+    _check(lib.tlq_selftest_bounded_wait(_ptr(workspace), workspace.numel() * workspace.element_size(), int(limit_cycles), st),
+           "tlq_selftest_bounded_wait")
+    return int(lib.tlq_read_status(_ptr(workspace), st))
 
 
 def tlq_stage_timing_enable(on: bool) -> None:

@@ -270,6 +270,26 @@ def test_device_errors_are_reported_not_raised_as_faults(tlq):
     assert tlq.tlq_kernel_launch_count() >= 0
 
 
+def test_bounded_wait_runs_out_and_is_reported(tlq):
+    """The device-side error path without a fault: a wait with a short limit on a barrier nothing arrives on gives
+    up, the status word says TLQ_ERR_TIMEOUT, and the very next search on the same workspace memory is normal."""
+    xb, wb, imp = wl.small_case(201, 200, 128, 96)
+    cfg = tlq.config(group_size=64, n_grid=4)
+    bufs = tlq.SearchBuffers(200, 128, 96, cfg, torch.device("cuda"))
+    assert tlq.tlq_selftest_bounded_wait(bufs.workspace, 1_000_000) == tlq.ERR_TIMEOUT
+    hdr = bufs.workspace[:256].view(torch.int32).cpu().numpy()
+    assert hdr[1] == 99 and hdr[4] == 1          # which wait gave up; the abort flag reached the other lanes
+    out = tlq.tlq_scale_search_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), torch.from_numpy(imp).cuda(), cfg, bufs)
+    assert tlq.tlq_read_status(out.workspace) == tlq.OK
+    ref = orc.scale_search(xb, wb, imp, "w4a16", 64, 4)
+    np.testing.assert_allclose(out.losses.cpu().numpy(), ref["losses"], rtol=LOSS_RTOL)
+    # host-side refusals of the self-test itself
+    import ctypes
+    assert tlq.lib.tlq_selftest_bounded_wait(bufs.workspace.data_ptr(), 16, 1000, None) == tlq.ERR_WORKSPACE
+    assert tlq.lib.tlq_selftest_bounded_wait(bufs.workspace.data_ptr(), 256, 0, None) == tlq.ERR_INVALID_ARG
+    assert tlq.lib.tlq_selftest_bounded_wait(bufs.workspace.data_ptr(), 256, 3_000_000_000, None) == tlq.ERR_INVALID_ARG
+
+
 # ----------------------------------------------------------------------------------- W8A8
 
 
