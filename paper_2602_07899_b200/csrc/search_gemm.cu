@@ -345,7 +345,7 @@ int launch_search_gemm_bf16(const uint16_t* X, const uint16_t* dW, const float* 
   const int sms = num_sms();
   if (sms <= 0) return TLQ_ERR_CUDA;
   const unsigned grid = (unsigned)(a.num_tiles < sms ? a.num_tiles : sms);
-  a.raster = make_raster(plan.mtiles, plan.otiles, sms, plan.N * plan.C1 * 2);
+  a.raster = make_raster(plan.mtiles, plan.otiles, sms, plan.N * plan.C1 * 2, BM);
   gemm_bf16_kernel<false><<<grid, kThreads, kSmemBytes, st>>>(tmA, tmB, tmB, a);
   return after_launch();
 }
@@ -369,7 +369,7 @@ int launch_apply_gemm_bf16(const uint16_t* X, const uint16_t* W, const uint16_t*
   const int sms = num_sms();
   if (sms <= 0) return TLQ_ERR_CUDA;
   const unsigned grid = (unsigned)(a.num_tiles < sms ? a.num_tiles : sms);
-  a.raster = make_raster(plan.mtiles, plan.otiles, sms, plan.N * plan.C1 * 2);
+  a.raster = make_raster(plan.mtiles, plan.otiles, sms, plan.N * plan.C1 * 2, BM);
   gemm_bf16_kernel<true><<<grid, kThreads, kSmemBytes, st>>>(tmA, tmW, tmD, a);
   return after_launch();
 }

@@ -445,7 +445,7 @@ int launch_search_gemm_i8(const uint16_t* X, const uint16_t* W, const int8_t* Xq
   const int sms = sm_count();
   if (sms <= 0) return TLQ_ERR_CUDA;
   const unsigned grid = (unsigned)(a.num_tiles < sms ? a.num_tiles : sms);
-  a.raster = make_raster(plan.mtiles, plan.otiles, sms, plan.N * plan.C1);
+  a.raster = make_raster(plan.mtiles, plan.otiles, sms, plan.N * plan.C1, BM);
   gemm_w8a8_kernel<0><<<grid, kThreads, kSmemBytes, st>>>(tmX, tmW, tmXq, tmWq, a);
   return after_launch();
 }
@@ -469,7 +469,7 @@ int launch_apply_gemm_i8(const int8_t* Xq, const int8_t* Wq, const float* t, con
   const int sms = sm_count();
   if (sms <= 0) return TLQ_ERR_CUDA;
   const unsigned grid = (unsigned)(a.num_tiles < sms ? a.num_tiles : sms);
-  a.raster = make_raster(plan.mtiles, plan.otiles, sms, plan.N * plan.C1);
+  a.raster = make_raster(plan.mtiles, plan.otiles, sms, plan.N * plan.C1, BM);
   gemm_w8a8_kernel<1><<<grid, kThreads, kSmemBytes, st>>>(tmXq, tmWq, tmXq, tmWq, a);
   return after_launch();
 }
@@ -505,7 +505,7 @@ int launch_search_gemm_dual_bf16(const uint16_t* Xq, const uint16_t* Xfp, const 
   const int sms = sm_count();
   if (sms <= 0) return TLQ_ERR_CUDA;
   const unsigned grid = (unsigned)(a.num_tiles < sms ? a.num_tiles : sms);
-  a.raster = make_raster(plan.mtiles, plan.otiles, sms, plan.N * plan.C1 * 2);
+  a.raster = make_raster(plan.mtiles, plan.otiles, sms, plan.N * plan.C1 * 2, BM);
   gemm_w8a8_kernel<2><<<grid, kThreads, kSmemBytes, st>>>(tmX, tmW, tmXq, tmD, a);
   return after_launch();
 }

@@ -263,7 +263,7 @@ int launch_search_gemm_bf16_wide(const uint16_t* X, const uint16_t* dW, const fl
   a.mpairs = ceil_div(plan.N, 2 * BM);
   a.otiles = plan.otiles;
   a.n_pad = plan.n_pad;
-  a.raster = make_raster(a.mpairs, a.otiles, sms, plan.N * plan.C1 * 2);
+  a.raster = make_raster(a.mpairs, a.otiles, sms, plan.N * plan.C1 * 2, 2 * BM);
   a.w_imp = w_imp; a.partials = partials; a.ptab = ptab; a.hdr = hdr; a.n_live = n_live;
   const int64_t tiles = (int64_t)plan.K * a.otiles * a.mpairs;
   const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
