@@ -6,6 +6,7 @@
 #include <nvtx3/nvToolsExt.h>
 
 #include "common.cuh"
+#include "l2part.cuh"
 
 namespace tlq {
 
@@ -345,6 +346,8 @@ static int search_impl(const void* X, const void* X_ref, int64_t N, int64_t C1, 
     Xg = L.Xc; wg = L.wc; n_live = L.live;
   }
   if (cfg->mode == TLQ_W4A16_ASYM_GROUP) {
+    // which L2 partition each SM sits next to: measured once per device, in the not yet written delta-weight region
+    const L2PartMap* l2map = l2_partition_map(L.dW, (size_t)K * C2 * C1 * sizeof(uint16_t), st);
     if ((rc = launch_fakequant_group(Wb, L.s, L.rs, K, C2, C1, cfg->group_size, cfg->w_bits, L.dW, nullptr, nullptr,
                                      nullptr, st)) != TLQ_OK)
       return rc;
@@ -358,7 +361,8 @@ static int search_impl(const void* X, const void* X_ref, int64_t N, int64_t C1, 
         return rc;
     } else if ((cfg->flags & TLQ_FLAG_GEMM_NARROW_TILES) || N <= 128) {
       if ((rc = launch_search_gemm_bf16(Xg, L.dW, wg, L.plan, L.partials, ptab, L.hdr, n_live, st)) != TLQ_OK) return rc;
-    } else if ((rc = launch_search_gemm_bf16_wide(Xg, L.dW, wg, L.plan, L.partials, ptab, L.hdr, n_live, st)) != TLQ_OK) {
+    } else if ((rc = launch_search_gemm_bf16_wide(Xg, L.dW, wg, L.plan, L.partials, ptab, L.hdr, n_live, l2map, st)) !=
+               TLQ_OK) {
       return rc;
     }
   } else {

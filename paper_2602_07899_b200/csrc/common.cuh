@@ -137,7 +137,9 @@ struct WorkspaceHeader {
   int32_t where;      // diagnostic: which wait gave up
   int32_t best_idx;   // device copy of the argmin
   int32_t reduce_done; // CTAs of the loss reduction that have finished (the header is zeroed by every call)
-  int32_t pad[60];
+  int32_t selftest;    // set by the bounded-wait self-test when its abort flag reached the other lanes
+  int32_t slot_count[2]; // tile-walk slots claimed so far in each L2 partition by the CTAs of the search GEMM
+  int32_t pad[57];
 };
 static_assert(sizeof(WorkspaceHeader) == 256, "header is 256 bytes");
 
@@ -211,10 +213,12 @@ int search_gemm_pair_capacity();
 int launch_search_gemm_bf16_pair(const uint16_t* X, const uint16_t* dW, const float* w_imp, const GemmPlan& plan,
                                  float* partials, float* ptab, WorkspaceHeader* hdr, const int32_t* n_live,
                                  cudaStream_t st);
-// search_gemm_wide.cu: the same search on 256-token x 256-channel tiles per CTA (weight tile shared by two halves)
+// search_gemm_wide.cu: the same search on 256-token x 256-channel tiles per CTA (weight tile shared by two halves);
+// l2map: the device's SM -> L2 partition table (l2part.cuh) or null
+struct L2PartMap;
 int launch_search_gemm_bf16_wide(const uint16_t* X, const uint16_t* dW, const float* w_imp, const GemmPlan& plan,
                                  float* partials, float* ptab, WorkspaceHeader* hdr, const int32_t* n_live,
-                                 cudaStream_t st);
+                                 const L2PartMap* l2map, cudaStream_t st);
 // Apply: Yq[N,C2] = X W^T - X dW^T (+bias), bf16 out
 int launch_apply_gemm_bf16(const uint16_t* X, const uint16_t* W, const uint16_t* dW, const uint16_t* bias,
                            int64_t N, int64_t C1, int64_t C2, uint16_t* Yq, WorkspaceHeader* hdr, cudaStream_t st);

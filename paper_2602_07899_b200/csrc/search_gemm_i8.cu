@@ -445,7 +445,11 @@ int launch_search_gemm_i8(const uint16_t* X, const uint16_t* W, const int8_t* Xq
   const int sms = sm_count();
   if (sms <= 0) return TLQ_ERR_CUDA;
   const unsigned grid = (unsigned)(a.num_tiles < sms ? a.num_tiles : sms);
-  a.raster = make_raster(plan.mtiles, plan.otiles, sms, plan.N * plan.C1, BM);
+  // Every candidate's int8 operands are read once and never again, so nothing is worth keeping in L2 between
+  // passes and what counts is how many distinct operand rows the CTAs of a wave share: always the blocked walk
+  // (16 token tiles x 9 output tiles: 15.6 MB per wave and pass on the 7B-class gate projection against 31.4 MB for
+  // all 64 token tiles x 2.3 output tiles).
+  a.raster = make_raster(plan.mtiles, plan.otiles, sms, (int64_t)1 << 40, BM);
   gemm_w8a8_kernel<0><<<grid, kThreads, kSmemBytes, st>>>(tmX, tmW, tmXq, tmWq, a);
   return after_launch();
 }

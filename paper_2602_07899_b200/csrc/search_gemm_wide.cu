@@ -14,6 +14,7 @@
 // Barriers: full[s] / empty[s] per stage, tfull (both accumulators complete), tempty[h] per half
 // (four epilogue warps).  Every wait is bounded.
 #include "common.cuh"
+#include "l2part.cuh"
 #include "umma.cuh"
 
 namespace tlq {
@@ -41,7 +42,9 @@ struct WideArgs {
   int64_t mpairs;          // 256-row token tiles
   int64_t otiles;
   int64_t n_pad;
-  TileRaster raster;       // over (mpairs, otiles)
+  bool blocked;            // walk by blocks of `block_a` token tiles (activations too large to stay in L2)
+  int block_a;
+  const L2PartMap* l2map;  // which L2 partition each SM sits next to (may be null or not yet measured)
   const float* w_imp;
   float* partials;         // [K][otiles*mtiles*4]
   float* ptab;             // [K][otiles][n_pad] or null
@@ -67,9 +70,15 @@ gemm_bf16_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
   auto tempty_bar = [&](int h) { return bar_base + 8u * (2 * kStages + 1 + h); };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + kStages * kStageBytes + 8 * (2 * kStages + 3));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  TileWalk* walk_sh = reinterpret_cast<TileWalk*>(smem_gen + kStages * kStageBytes + 128);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
+  int64_t n_tokens = args.N, mpairs = args.mpairs;
+  if (args.n_live != nullptr) {
+    n_tokens = *args.n_live;
+    mpairs = (n_tokens + 2 * BM - 1) / (2 * BM);
+  }
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       ptx::mbar_init(full_bar(s), 1);
@@ -82,24 +91,16 @@ gemm_bf16_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     ptx::fence_barrier_init();
     ptx::prefetch_tensormap(&tmA);
     ptx::prefetch_tensormap(&tmB);
+    // this CTA's share of the tiles: its L2 partition's token tiles when the partitions are known
+    make_tile_walk(args.l2map, args.hdr, (int)mpairs, (int)args.otiles, args.K, args.blocked, args.block_a, *walk_sh);
   }
   if (warp == 1) ptx::tmem_alloc(ptx::smem_u32(tmem_slot), kTmemCols);
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-
+  const TileWalk walk = *walk_sh;
   const int num_kb = args.num_kb;
-  int64_t n_tokens = args.N, mpairs = args.mpairs;
-  TileRaster raster = args.raster;
-  if (args.n_live != nullptr) {
-    n_tokens = *args.n_live;
-    mpairs = (n_tokens + 2 * BM - 1) / (2 * BM);
-    raster.mtiles = (int)mpairs;
-    if (raster.b == 1) raster.a = mpairs > 0 ? (int)mpairs : 1;
-  }
-  const int64_t tiles_per_k = args.otiles * mpairs;
-  const int64_t num_tiles = (int64_t)args.K * tiles_per_k;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -107,10 +108,9 @@ gemm_bf16_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-        const int k = (int)(tile / tiles_per_k);
-        int mp, ot;
-        raster.decode(tile - (int64_t)k * tiles_per_k, mp, ot);
+      for (int64_t tile = walk.first; tile < walk.count && ok; tile += walk.stride) {
+        int k, mp, ot;
+        walk.decode(tile, k, mp, ot);
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!ptx::mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
             report_timeout(args.hdr, 31);
@@ -132,7 +132,7 @@ gemm_bf16_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
       uint32_t phase = 0;
       int64_t it = 0;
       bool ok = true;
-      for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+      for (int64_t tile = walk.first; tile < walk.count && ok; tile += walk.stride, ++it) {
         const uint32_t drained_phase = (uint32_t)(it & 1) ^ 1u;     // halves were drained once per earlier tile
         for (int kb = 0; kb < num_kb && ok; ++kb) {
           if (!ptx::mbar_wait(full_bar(stage), phase, abort_flag)) {
@@ -172,10 +172,9 @@ gemm_bf16_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     const int quarter = warp & 3;
     const int row_in_half = quarter * 32 + lane;
     int64_t it = 0;
-    for (int64_t tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
-      const int k = (int)(tile / tiles_per_k);
-      int mp, ot;
-      raster.decode(tile - (int64_t)k * tiles_per_k, mp, ot);
+    for (int64_t tile = walk.first; tile < walk.count; tile += walk.stride, ++it) {
+      int k, mp, ot;
+      walk.decode(tile, k, mp, ot);
       if (!ptx::mbar_wait(tfull_bar, (uint32_t)(it & 1), abort_flag)) {
         if (lane == 0) report_timeout(args.hdr, 34);
         break;
@@ -237,7 +236,7 @@ int wide_sm_count() { return device_sm_count(); }
 
 int launch_search_gemm_bf16_wide(const uint16_t* X, const uint16_t* dW, const float* w_imp, const GemmPlan& plan,
                                  float* partials, float* ptab, WorkspaceHeader* hdr, const int32_t* n_live,
-                                 cudaStream_t st) {
+                                 const L2PartMap* l2map, cudaStream_t st) {
   static OncePerDevice once;
   const int rc_cfg = once_per_device(once, [] {
     return cudaFuncSetAttribute(gemm_bf16_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
@@ -263,10 +262,17 @@ int launch_search_gemm_bf16_wide(const uint16_t* X, const uint16_t* dW, const fl
   a.mpairs = ceil_div(plan.N, 2 * BM);
   a.otiles = plan.otiles;
   a.n_pad = plan.n_pad;
-  a.raster = make_raster(a.mpairs, a.otiles, sms, plan.N * plan.C1 * 2, 2 * BM);
+  const TileRaster shape = make_raster(a.mpairs, a.otiles, sms, plan.N * plan.C1 * 2, 2 * BM);
+  a.blocked = shape.b != 1;
+  a.block_a = 2048 / (2 * BM);
   a.w_imp = w_imp; a.partials = partials; a.ptab = ptab; a.hdr = hdr; a.n_live = n_live;
   const int64_t tiles = (int64_t)plan.K * a.otiles * a.mpairs;
   const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
+  // The partition-aware walk needs one CTA on every SM and enough tiles for the split to balance.  It is for
+  // activations that can stay in L2 (measured on the 7B-class layer: HBM bytes of the q / k / gate launches 1677 /
+  // 318 / 9700 MB -> 644 / 132 / 5240 MB); where they cannot, splitting the tokens only shortens the weight block a
+  // wave shares (18944-channel down-projection: 24.5 -> 45 GB), so the blocked walk stays whole.
+  a.l2map = (grid == (unsigned)sms && tiles >= 8 * (int64_t)sms && !a.blocked) ? l2map : nullptr;
   gemm_bf16_wide_kernel<<<grid, kThreads, kSmemBytes, st>>>(tmA, tmB, a);
   return after_launch();
 }

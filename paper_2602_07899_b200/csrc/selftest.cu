@@ -28,7 +28,7 @@ __global__ void bounded_wait_selftest_kernel(WorkspaceHeader* hdr, long long lim
   }
   __syncthreads();
   // the second lane sees the flag the first one left behind: how the other roles of a CTA learn of a timeout
-  if (threadIdx.x == 1 && abort_flag != 0) hdr->pad[0] = 1;
+  if (threadIdx.x == 1 && abort_flag != 0) hdr->selftest = 1;
 }
 
 int launch_bounded_wait_selftest(WorkspaceHeader* hdr, long long limit_cycles, cudaStream_t st) {

@@ -20,11 +20,13 @@ from oracle import tlq_oracle as orc
 from paper_2602_07899_b200 import workloads as wl
 
 LOSS_RTOL = 2e-3
-# Measured distance between the CUDA path's losses and the oracle's at full size: up to 4e-5 relative in the group
-# mode (bf16 rounding of the delta-weight operand, fp32 accumulation), 5e-6 in the symmetric modes, of which at
-# most 3e-5 differs between the candidates of one linear; an oracle gap below this floor would make "identical
-# argmin" a coin toss rather than a property of the method.
-GAP_FLOOR = 1e-4
+# What decides whether the CUDA path can reproduce an argmin is how differently its arithmetic (bf16 rounding of the
+# delta-weight operand, fp32 accumulation in tensor memory) shifts the losses of the oracle's two best candidates.
+# Measured on every stored linear: that difference is at most 2.3e-5 relative (the 256-row key / value projections of
+# the 2B-class sweep) and at most 6e-6 for projections of 1536 rows and more, never more than a seventh of the
+# oracle's own gap.  An oracle gap below the floor would make "identical argmin" a coin toss rather than a property
+# of the method.
+GAP_FLOOR = 4e-5
 GOLDEN_DIR = os.path.join(os.path.dirname(__file__), "golden", "fullsize")
 ORDER = {n: i for i, n in enumerate(("q", "k", "v", "o", "gate", "up", "down"))}
 

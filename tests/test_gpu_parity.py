@@ -724,3 +724,27 @@ def test_row_quantizers_on_very_wide_rows(tlq):
     qx, t = orc.quantize_activations_token_sym(xb, s_np)
     assert np.array_equal(out["codes"].cpu().numpy(), qw) and np.array_equal(out["steps"].cpu().numpy(), u)
     assert np.array_equal(codes.cpu().numpy(), qx) and np.array_equal(steps.cpu().numpy(), t)
+
+
+def test_search_with_the_l2_partition_aware_tile_walk(tlq):
+    """Large enough for the 256-token kernel to run one CTA per SM with the tile space split between the two L2
+    partitions (when the device's partition table could be measured): same results, every slot claimed once."""
+    xb, wb, imp = wl.small_case(211, 2048, 512, 2048)
+    ref = orc.scale_search(xb, wb, imp, "w4a16", 128, 20)
+    for _ in range(2):      # the first large call on a device also measures the table
+        got = run_search(tlq, xb, wb, imp)
+        check_against_oracle(got, ref, 20)
+    cfg = tlq.config()
+    out = tlq.tlq_scale_search_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), torch.from_numpy(imp).cuda(), cfg)
+    hdr = out.workspace[:256].view(torch.int32).cpu().numpy()
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    assert hdr[0] == 0 and int(hdr[5]) + int(hdr[6]) in (0, sms), hdr[:8]
+    print("tile-walk slots claimed per L2 partition:", int(hdr[5]), int(hdr[6]))
+    # token skipping on top: the live token count, and with it the split, is only known on the device
+    imp2 = imp.copy()
+    imp2[np.random.default_rng(3).random(2048) < 0.4] = 0.0
+    ref2 = orc.scale_search(xb, wb, imp2, "w4a16", 128, 20)
+    cfg2 = tlq.config(flags=tlq.FLAG_SKIP_ZERO_WEIGHT_TOKENS)
+    out2 = tlq.tlq_scale_search_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), torch.from_numpy(imp2).cuda(), cfg2)
+    np.testing.assert_allclose(out2.losses.cpu().numpy(), ref2["losses"], rtol=LOSS_RTOL)
+    assert_same_argmin(int(out2.best_idx.item()), ref2)
