@@ -190,6 +190,10 @@ int tlq_quantize_activations(const void* X, const void* s, int64_t N, int64_t C1
  *   best_idx [1] int32, losses [K] fp64, s_best [C1] bf16 (the winning scale),
  *   per_token_err [K,N] fp32 or NULL (e_{k,n}).
  * The workspace holds the operands of all K candidates; its status word is reset by this call.
+ * Group mode: the first call on a device whose K x C2 x C1 delta-weight region is at least 35 MB also enqueues, once,
+ * a measurement of about a millisecond (which half of the L2 each SM sits next to; it uses that region before
+ * anything else is written there) and looks up a device symbol's address; make that first call outside of any
+ * stream capture.  Results do not depend on it, only the order in which tiles are visited.
  */
 size_t tlq_scale_search_workspace_bytes(int64_t N, int64_t C1, int64_t C2, const tlq_config* cfg);
 int tlq_scale_search_layer(const void* X, int64_t N, int64_t C1, const void* W, int64_t C2,
