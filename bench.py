@@ -330,13 +330,14 @@ def stage_report(tlq, cfgr, lins, leg, live_frac, peaks):
 
 
 def roofline_record(kernel, i8, achieved, peaks, clocks, traffic, launches_timed, share, lib_int8=None):
-    """Roofline of the fused search GEMM.  The comparator follows the run's own clock record: a region that
-    ran into the power cap (or whose median SM clock sat below 85 % of the maximum) is compared with the
-    sustained library rate, a short region at full clock with the burst rate.  int8 takes the measured bf16
+    """Roofline of the fused search GEMM.  The comparator follows the run's own clock record: a region whose
+    median SM clock sat below 85 % of the maximum (the power cap of a long run) is compared with the sustained
+    library rate, a short region at full clock with the burst rate.  int8 takes the measured bf16
     peak times the nominal int8 : bf16 ratio of 2."""
     ratio = 2.0 if i8 else 1.0
     sm, mx = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
-    capped = "sw_power_cap" in clocks.get("reasons", []) or (sm is not None and mx and sm < 0.85 * mx) or sm is None
+    # the median clock decides (the power-cap reason alone also shows up for a moment when a 300 W run starts)
+    capped = sm is None or not mx or sm < 0.85 * mx
     comparator = "sustained" if capped else "burst"
     peak = peaks["bf16_sustained" if capped else "bf16_burst"] * ratio
     nominal = 2250.0 * ratio
