@@ -32,28 +32,51 @@ size_t l2_partition_scratch_bytes();
 const L2PartMap* l2_partition_map(void* scratch, size_t scratch_bytes, cudaStream_t st);
 
 // This CTA's share of a (candidate, output tile, token tile) space.
+//
+// Whole grid (part < 0): items are (candidate, position in the raster over all token and output tiles).
+// One L2 partition (part 0 or 1): the token tiles are cut between the partitions in proportion to their SM counts.
+// The exact proportion is rarely a whole number of tiles (72 of 148 SMs want 15.57 of 32 tiles), and rounding it
+// would leave one partition several percent more rounds than the other, so the cut moves from candidate to
+// candidate: after k candidates partition 0 has had floor(k * mtiles * n0 / n) token tiles in total, i.e. 15 or 16
+// per candidate in the right mix.  Inside a candidate the partition walks its token tiles fastest, then the output
+// tiles.
 struct TileWalk {
   int first, stride;        // work items first, first + stride, ... below `count`
-  int m_first, m_count;     // token tiles [m_first, m_first + m_count) of this CTA's partition
-  int64_t count;            // K * otiles * m_count
-  int64_t tiles_per_k;      // otiles * m_count
-  TileRaster raster;        // over (m_count, otiles)
+  int part;                 // -1: the whole grid shares one walk
+  int mtiles, otiles;
+  int n0, n;                // SMs of partition 0, SMs in total
+  int64_t count;            // items of this walk
+  TileRaster raster;        // whole-grid walk only: over (mtiles, otiles)
+
+  __device__ int64_t tiles0_before(int k) const { return ((int64_t)k * mtiles * n0) / n; }   // partition 0's token tiles
+  __device__ int64_t base(int k) const {            // items before candidate k
+    if (part < 0) return (int64_t)k * otiles * mtiles;
+    const int64_t t0 = tiles0_before(k);
+    return (int64_t)otiles * (part == 0 ? t0 : (int64_t)k * mtiles - t0);
+  }
+  // `k` is the caller's running candidate: items only ever increase, so it is advanced, never searched
   __device__ void decode(int64_t item, int& k, int& mt, int& ot) const {
-    k = (int)(item / tiles_per_k);
-    int ml;
-    raster.decode(item - (int64_t)k * tiles_per_k, ml, ot);
-    mt = m_first + ml;
+    while (item >= base(k + 1)) ++k;
+    const int64_t r = item - base(k);
+    if (part < 0) {
+      raster.decode(r, mt, ot);
+    } else {
+      const int cut = (int)(tiles0_before(k + 1) - tiles0_before(k));
+      const int mc = part == 0 ? cut : mtiles - cut;
+      ot = (int)(r / mc);
+      mt = (part == 0 ? 0 : cut) + (int)(r - (int64_t)ot * mc);
+    }
   }
 };
 
 // Called by ONE thread of every CTA of the grid, exactly once per launch.  `mtiles` token tiles, `otiles` output
-// tiles, K candidates; `blocked` says whether the walk inside a partition goes by blocks of `block_a` token tiles.
-// `hdr->slot_count` must have been zeroed before the launch.
+// tiles, K candidates; `blocked` says whether the whole-grid walk goes by blocks of `block_a` token tiles (then the
+// partitions are not used: see the launcher).  `hdr->slot_count` must have been zeroed before the launch.
 __device__ inline void make_tile_walk(const L2PartMap* map, WorkspaceHeader* hdr, int mtiles, int otiles, int K,
                                       bool blocked, int block_a, TileWalk& w) {
   const int grid = (int)gridDim.x;
   int part = -1, rank = (int)blockIdx.x, n_part = grid;
-  if (map != nullptr && map->valid != 0 && map->n_sms == grid && mtiles >= 4) {
+  if (map != nullptr && map->valid != 0 && map->n_sms == grid && mtiles >= 4 && !blocked) {
     unsigned smid;
     asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
     int p = smid < (unsigned)kMaxSmIds ? (int)map->part[smid] : 0;
@@ -71,26 +94,21 @@ __device__ inline void make_tile_walk(const L2PartMap* map, WorkspaceHeader* hdr
   }
   w.first = rank;
   w.stride = n_part;
-  if (part < 0) {
-    w.m_first = 0;
-    w.m_count = mtiles;
-  } else {
-    int m0 = (int)(((int64_t)mtiles * map->count[0] + grid / 2) / grid);     // token tiles in proportion to the SMs
-    m0 = m0 < 1 ? 1 : (m0 > mtiles - 1 ? mtiles - 1 : m0);
-    w.m_first = part == 0 ? 0 : m0;
-    w.m_count = part == 0 ? m0 : mtiles - m0;
-  }
-  w.tiles_per_k = (int64_t)otiles * w.m_count;
-  w.count = (int64_t)K * w.tiles_per_k;
-  w.raster.mtiles = w.m_count;
+  w.part = part;
+  w.mtiles = mtiles;
+  w.otiles = otiles;
+  w.n0 = part < 0 ? 1 : map->count[0];
+  w.n = part < 0 ? 1 : grid;
+  w.raster.mtiles = mtiles;
   w.raster.otiles = otiles;
   if (blocked) {
     w.raster.a = block_a;
-    w.raster.b = n_part / block_a > 0 ? n_part / block_a : 1;
+    w.raster.b = grid / block_a > 0 ? grid / block_a : 1;
   } else {
-    w.raster.a = w.m_count > 0 ? w.m_count : 1;
+    w.raster.a = mtiles > 0 ? mtiles : 1;
     w.raster.b = 1;
   }
+  w.count = w.base(K);
 }
 
 }  // namespace tlq

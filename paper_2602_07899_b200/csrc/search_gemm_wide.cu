@@ -108,8 +108,9 @@ gemm_bf16_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
+      int k = 0;
       for (int64_t tile = walk.first; tile < walk.count && ok; tile += walk.stride) {
-        int k, mp, ot;
+        int mp, ot;
         walk.decode(tile, k, mp, ot);
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!ptx::mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
@@ -172,8 +173,9 @@ gemm_bf16_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     const int quarter = warp & 3;
     const int row_in_half = quarter * 32 + lane;
     int64_t it = 0;
+    int k = 0;
     for (int64_t tile = walk.first; tile < walk.count; tile += walk.stride, ++it) {
-      int k, mp, ot;
+      int mp, ot;
       walk.decode(tile, k, mp, ot);
       if (!ptx::mbar_wait(tfull_bar, (uint32_t)(it & 1), abort_flag)) {
         if (lane == 0) report_timeout(args.hdr, 34);
