@@ -22,6 +22,10 @@
  *    to the int32 status word at byte 0 of the workspace; tlq_read_status() synchronises the stream
  *    and returns it.
  *  - There is no CPU fallback: without a CUDA device every compute call returns TLQ_ERR_CUDA.
+ *  - Every call acts on the device that is current when it is made; the few pieces of host-side state the library
+ *    keeps (kernel attributes, SM counts, addresses of its built-in device arrays) are kept per device, so one process
+ *    may drive several GPUs.  Calls are not synchronised against each other: host threads that share a device, or a
+ *    workspace, must take turns.
  */
 #ifndef TLQ_H_
 #define TLQ_H_
