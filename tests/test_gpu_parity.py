@@ -726,10 +726,13 @@ def test_row_quantizers_on_very_wide_rows(tlq):
     assert np.array_equal(codes.cpu().numpy(), qx) and np.array_equal(steps.cpu().numpy(), t)
 
 
-def test_search_with_the_l2_partition_aware_tile_walk(tlq):
+@pytest.mark.parametrize("n,c2", [(2048, 2048), (2304, 1792), (2100, 2000)])
+def test_search_with_the_l2_partition_aware_tile_walk(tlq, n, c2):
     """Large enough for the 256-token kernel to run one CTA per SM with the tile space split between the two L2
-    partitions (when the device's partition table could be measured): same results, every slot claimed once."""
-    xb, wb, imp = wl.small_case(211, 2048, 512, 2048)
+    partitions (when the device's partition table could be measured): same results, every slot claimed once.
+    The whole per-token table is compared, so a tile that no CTA visited would show as a missing share of 256
+    tokens' errors.  Even, odd and ragged tile counts (the cut between the partitions moves with the candidate)."""
+    xb, wb, imp = wl.small_case(211, n, 512, c2)
     ref = orc.scale_search(xb, wb, imp, "w4a16", 128, 20)
     for _ in range(2):      # the first large call on a device also measures the table
         got = run_search(tlq, xb, wb, imp)
@@ -742,7 +745,7 @@ def test_search_with_the_l2_partition_aware_tile_walk(tlq):
     print("tile-walk slots claimed per L2 partition:", int(hdr[5]), int(hdr[6]))
     # token skipping on top: the live token count, and with it the split, is only known on the device
     imp2 = imp.copy()
-    imp2[np.random.default_rng(3).random(2048) < 0.4] = 0.0
+    imp2[np.random.default_rng(3).random(n) < 0.4] = 0.0
     ref2 = orc.scale_search(xb, wb, imp2, "w4a16", 128, 20)
     cfg2 = tlq.config(flags=tlq.FLAG_SKIP_ZERO_WEIGHT_TOKENS)
     out2 = tlq.tlq_scale_search_layer(dev_bf16(tlq, xb), dev_bf16(tlq, wb), torch.from_numpy(imp2).cuda(), cfg2)
