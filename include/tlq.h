@@ -245,6 +245,17 @@ int tlq_read_status(const void* workspace, void* stream);
 int tlq_selftest_bounded_wait(void* workspace, size_t workspace_bytes, int64_t limit_cycles, void* stream);
 
 /*
+ * Diagnostic, host only (the paper has no counterpart; no device is touched): the order in which the persistent CTAs
+ * of the fused bf16 GEMM visit the (candidate, output tile, token tile) space, replayed on the host.  With n1 = 0
+ * it is the walk of a grid of n0 CTAs (blocked != 0: by blocks of block_a token tiles); with n1 > 0 the walk of
+ * n0 + n1 CTAs split over the two L2 partitions (n0 and n1 SMs; token tiles cut between them, blocked must be 0,
+ * mtiles >= 4).  Every visit adds one to visits[(k * otiles + ot) * mtiles + mt] (HOST array of K * otiles * mtiles
+ * int32, zeroed by the caller): a correct walk leaves every entry at exactly 1.
+ */
+int tlq_debug_tile_walk(int64_t mtiles, int64_t otiles, int32_t K, int32_t n0, int32_t n1, int32_t blocked,
+                        int32_t block_a, int32_t* visits /* host */);
+
+/*
  * Per-stage device timing of tlq_scale_search_layer, for benchmarks.  While enabled, every search call
  * records CUDA events on its stream between its stages (event sets come from a pool of 512 created on
  * first use; further calls are not recorded).  _drain() synchronises on the recorded events, writes

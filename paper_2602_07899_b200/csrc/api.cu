@@ -182,7 +182,7 @@ const char* tlq_status_string(int status) {
   }
 }
 
-int tlq_version(void) { return 1005; }   // 1.5: bounded-wait self-test
+int tlq_version(void) { return 1006; }   // 1.6: bounded-wait self-test, tile-walk check
 
 int64_t tlq_kernel_launch_count(void) { return (int64_t)g_launch_count; }
 
@@ -494,6 +494,32 @@ int tlq_selftest_bounded_wait(void* workspace, size_t workspace_bytes, int64_t l
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   TLQ_CUDA_TRY(cudaMemsetAsync(workspace, 0, sizeof(WorkspaceHeader), st));
   return launch_bounded_wait_selftest(reinterpret_cast<WorkspaceHeader*>(workspace), (long long)limit_cycles, st);
+}
+
+int tlq_debug_tile_walk(int64_t mtiles, int64_t otiles, int32_t K, int32_t n0, int32_t n1, int32_t blocked,
+                        int32_t block_a, int32_t* visits) {
+  if (visits == nullptr) return TLQ_ERR_INVALID_ARG;
+  if (mtiles < 1 || otiles < 1 || K < 1 || K > TLQ_MAX_GRID || n0 < 1 || n1 < 0 || block_a < 1 ||
+      mtiles > 0x7FFFFF || otiles > 0x7FFFFF)
+    return TLQ_ERR_SHAPE;
+  const bool split = n1 > 0;
+  if (split && (blocked != 0 || mtiles < 4 || n0 * 4 < n0 + n1 || n1 * 4 < n0 + n1)) return TLQ_ERR_UNSUPPORTED;
+  const int grid = n0 + n1;
+  for (int part = split ? 0 : -1; part < (split ? 2 : 0); ++part) {
+    const int n_part = split ? (part == 0 ? n0 : n1) : grid;
+    for (int rank = 0; rank < n_part; ++rank) {
+      TileWalk w;
+      fill_tile_walk(w, part, rank, n_part, (int)mtiles, (int)otiles, K, blocked != 0, block_a, n0, grid);
+      int k = 0;
+      for (int64_t item = w.first; item < w.count; item += w.stride) {
+        int mt, ot;
+        w.decode(item, k, mt, ot);
+        if (k < 0 || k >= K || mt < 0 || mt >= mtiles || ot < 0 || ot >= otiles) return TLQ_ERR_INVALID_ARG;
+        visits[((int64_t)k * otiles + ot) * mtiles + mt] += 1;
+      }
+    }
+  }
+  return TLQ_OK;
 }
 
 int tlq_stage_timing_enable(int on) {

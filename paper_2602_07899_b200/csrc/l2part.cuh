@@ -48,14 +48,14 @@ struct TileWalk {
   int64_t count;            // items of this walk
   TileRaster raster;        // whole-grid walk only: over (mtiles, otiles)
 
-  __device__ int64_t tiles0_before(int k) const { return ((int64_t)k * mtiles * n0) / n; }   // partition 0's token tiles
-  __device__ int64_t base(int k) const {            // items before candidate k
+  __host__ __device__ int64_t tiles0_before(int k) const { return ((int64_t)k * mtiles * n0) / n; }   // partition 0's token tiles
+  __host__ __device__ int64_t base(int k) const {            // items before candidate k
     if (part < 0) return (int64_t)k * otiles * mtiles;
     const int64_t t0 = tiles0_before(k);
     return (int64_t)otiles * (part == 0 ? t0 : (int64_t)k * mtiles - t0);
   }
   // `k` is the caller's running candidate: items only ever increase, so it is advanced, never searched
-  __device__ void decode(int64_t item, int& k, int& mt, int& ot) const {
+  __host__ __device__ void decode(int64_t item, int& k, int& mt, int& ot) const {
     while (item >= base(k + 1)) ++k;
     const int64_t r = item - base(k);
     if (part < 0) {
@@ -68,6 +68,29 @@ struct TileWalk {
     }
   }
 };
+
+// The walk of slot `rank` of `n_part` in partition `part` (-1: slot `rank` of a whole grid of `grid` CTAs).  Pure
+// integer arithmetic, shared by the kernels and by the host-side coverage check (tlq_debug_tile_walk).
+__host__ __device__ inline void fill_tile_walk(TileWalk& w, int part, int rank, int n_part, int mtiles, int otiles,
+                                               int K, bool blocked, int block_a, int n0, int grid) {
+  w.first = rank;
+  w.stride = n_part;
+  w.part = part;
+  w.mtiles = mtiles;
+  w.otiles = otiles;
+  w.n0 = part < 0 ? 1 : n0;
+  w.n = part < 0 ? 1 : grid;
+  w.raster.mtiles = mtiles;
+  w.raster.otiles = otiles;
+  if (blocked) {
+    w.raster.a = block_a;
+    w.raster.b = grid / block_a > 0 ? grid / block_a : 1;
+  } else {
+    w.raster.a = mtiles > 0 ? mtiles : 1;
+    w.raster.b = 1;
+  }
+  w.count = w.base(K);
+}
 
 // Called by ONE thread of every CTA of the grid, exactly once per launch.  `mtiles` token tiles, `otiles` output
 // tiles, K candidates; `blocked` says whether the whole-grid walk goes by blocks of `block_a` token tiles (then the
@@ -92,23 +115,7 @@ __device__ inline void make_tile_walk(const L2PartMap* map, WorkspaceHeader* hdr
       hdr->status = TLQ_ERR_TIMEOUT;
     }
   }
-  w.first = rank;
-  w.stride = n_part;
-  w.part = part;
-  w.mtiles = mtiles;
-  w.otiles = otiles;
-  w.n0 = part < 0 ? 1 : map->count[0];
-  w.n = part < 0 ? 1 : grid;
-  w.raster.mtiles = mtiles;
-  w.raster.otiles = otiles;
-  if (blocked) {
-    w.raster.a = block_a;
-    w.raster.b = grid / block_a > 0 ? grid / block_a : 1;
-  } else {
-    w.raster.a = mtiles > 0 ? mtiles : 1;
-    w.raster.b = 1;
-  }
-  w.count = w.base(K);
+  fill_tile_walk(w, part, rank, n_part, mtiles, otiles, K, blocked, block_a, part < 0 ? 1 : map->count[0], grid);
 }
 
 }  // namespace tlq

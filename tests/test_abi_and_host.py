@@ -31,7 +31,7 @@ def test_every_declared_symbol_is_exported(tlq):
     for n in names:
         assert hasattr(tlq.lib, n), n
     assert sorted(tlq.EXPORTS) == names
-    assert tlq.lib.tlq_version() == 1005
+    assert tlq.lib.tlq_version() == 1006
     assert tlq.status_string(0) == "ok" and "workspace" in tlq.status_string(tlq.ERR_WORKSPACE)
 
 
@@ -124,3 +124,32 @@ def test_oracle_never_imports_the_cuda_path():
         if fn.endswith(".py"):
             text = open(os.path.join(ROOT, "paper_2602_07899_b200", fn)).read()
             assert not re.search(r"^\s*(from|import)\s+oracle", text, flags=re.M), fn
+
+
+def test_tile_walk_visits_every_tile_exactly_once(tlq):
+    """The order in which the persistent CTAs of the fused GEMM take their tiles, replayed on the host: whole grid
+    (plain and blocked) and split over two L2 partitions of unequal size, whose token cut moves from candidate to
+    candidate.  Every (candidate, output tile, token tile) must be visited exactly once."""
+    import numpy as np
+    for mtiles, otiles, K in ((32, 74, 20), (32, 2, 20), (9, 7, 20), (4, 1, 1), (5, 3, 64), (64, 116, 3)):
+        for n0, n1 in ((72, 76), (70, 78), (74, 74), (40, 108)):
+            v = tlq.tlq_debug_tile_walk(mtiles, otiles, K, n0, n1)
+            assert v.min() == 1 and v.max() == 1, (mtiles, otiles, K, n0, n1)
+        for grid in (148, 7, 1):
+            assert np.all(tlq.tlq_debug_tile_walk(mtiles, otiles, K, grid) == 1)
+            assert np.all(tlq.tlq_debug_tile_walk(mtiles, otiles, K, grid, blocked=True, block_a=8) == 1)
+            assert np.all(tlq.tlq_debug_tile_walk(mtiles, otiles, K, grid, blocked=True, block_a=16) == 1)
+    # the partitions' shares follow their SM counts: both need about the same number of rounds
+    mt, ot, K, n0, n1 = 32, 74, 20, 72, 76
+    c0 = (K * mt * n0) // (n0 + n1)                  # token tiles of partition 0 summed over the candidates
+    rounds0 = -(-c0 * ot // n0)
+    rounds1 = -(-(K * mt - c0) * ot // n1)
+    assert abs(rounds0 - rounds1) <= 1
+    # refusals: a split needs an unblocked walk, four token tiles and partitions of comparable size
+    v = np.zeros(4 * 4, dtype=np.int32)
+    args = v.ctypes.data_as(__import__("ctypes").c_void_p)
+    assert tlq.lib.tlq_debug_tile_walk(4, 4, 1, 72, 76, 1, 8, args) == tlq.ERR_UNSUPPORTED
+    assert tlq.lib.tlq_debug_tile_walk(3, 4, 1, 72, 76, 0, 8, args) == tlq.ERR_UNSUPPORTED
+    assert tlq.lib.tlq_debug_tile_walk(4, 4, 1, 10, 138, 0, 8, args) == tlq.ERR_UNSUPPORTED
+    assert tlq.lib.tlq_debug_tile_walk(4, 4, 0, 72, 76, 0, 8, args) == tlq.ERR_SHAPE
+    assert tlq.lib.tlq_debug_tile_walk(4, 4, 1, 72, 76, 0, 8, None) == tlq.ERR_INVALID_ARG
