@@ -255,6 +255,12 @@ int tlq_selftest_bounded_wait(void* workspace, size_t workspace_bytes, int64_t l
 int tlq_debug_tile_walk(int64_t mtiles, int64_t otiles, int32_t K, int32_t n0, int32_t n1, int32_t blocked,
                         int32_t block_a, int32_t* visits /* host */);
 
+/* The same replay for the tile-resident kernels (symmetric modes, two-stream search): `grid` persistent CTAs, each
+ * keeping an output tile for all K candidates, the tiles of the last partial wave split by candidates over the idle
+ * CTAs; blocked != 0 walks the tiles in blocks of 16 token tiles.  Same `visits` layout and meaning. */
+int tlq_debug_resident_walk(int64_t mtiles, int64_t otiles, int32_t K, int32_t grid, int32_t blocked,
+                            int32_t* visits /* host */);
+
 /*
  * Per-stage device timing of tlq_scale_search_layer, for benchmarks.  While enabled, every search call
  * records CUDA events on its stream between its stages (event sets come from a pool of 512 created on

@@ -522,6 +522,27 @@ int tlq_debug_tile_walk(int64_t mtiles, int64_t otiles, int32_t K, int32_t n0, i
   return TLQ_OK;
 }
 
+int tlq_debug_resident_walk(int64_t mtiles, int64_t otiles, int32_t K, int32_t grid, int32_t blocked, int32_t* visits) {
+  if (visits == nullptr) return TLQ_ERR_INVALID_ARG;
+  if (mtiles < 1 || otiles < 1 || K < 1 || K > TLQ_MAX_GRID || grid < 1 || mtiles * otiles > 0x7FFFFFFF)
+    return TLQ_ERR_SHAPE;
+  const int num_tiles = (int)(mtiles * otiles);
+  const TileRaster raster = make_raster(mtiles, otiles, grid, blocked ? ((int64_t)1 << 40) : 0, 128);
+  const TailSplit split = make_tail_split(num_tiles, grid, K);
+  for (int cta = 0; cta < grid; ++cta) {
+    for (int w = cta;; w += grid) {
+      int tile, k0, k1;
+      if (!work_item(split, w, K, tile, k0, k1)) break;
+      int mt, ot;
+      raster.decode(tile, mt, ot);
+      if (tile < 0 || tile >= num_tiles || mt < 0 || mt >= mtiles || ot < 0 || ot >= otiles || k0 < 0 || k1 > K)
+        return TLQ_ERR_INVALID_ARG;
+      for (int k = k0; k < k1; ++k) visits[((int64_t)k * otiles + ot) * mtiles + mt] += 1;
+    }
+  }
+  return TLQ_OK;
+}
+
 int tlq_stage_timing_enable(int on) {
   g_timing_on = on != 0;
   g_calls = 0;

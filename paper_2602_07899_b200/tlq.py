@@ -31,7 +31,7 @@ EXPORTS = (
     "tlq_status_string", "tlq_version", "tlq_token_importance", "tlq_scale_candidates_workspace_bytes",
     "tlq_scale_candidates", "tlq_scale_candidates_noalloc", "tlq_quantize_weights", "tlq_pack_codes4", "tlq_quantize_activations", "tlq_scale_search_workspace_bytes", "tlq_scale_search_layer", "tlq_scale_search_layer_two_stream",
     "tlq_apply_layer_workspace_bytes", "tlq_apply_layer", "tlq_read_status", "tlq_stage_timing_enable",
-    "tlq_stage_timing_drain", "tlq_kernel_launch_count", "tlq_selftest_bounded_wait", "tlq_debug_tile_walk",
+    "tlq_stage_timing_drain", "tlq_kernel_launch_count", "tlq_selftest_bounded_wait", "tlq_debug_tile_walk", "tlq_debug_resident_walk",
 )
 
 
@@ -96,6 +96,8 @@ def _load() -> ctypes.CDLL:
     lib.tlq_selftest_bounded_wait.restype = i32
     lib.tlq_debug_tile_walk.argtypes = [i64, i64, i32, i32, i32, i32, i32, vp]
     lib.tlq_debug_tile_walk.restype = i32
+    lib.tlq_debug_resident_walk.argtypes = [i64, i64, i32, i32, i32, vp]
+    lib.tlq_debug_resident_walk.restype = i32
     lib.tlq_stage_timing_enable.argtypes = [i32]
     lib.tlq_stage_timing_drain.argtypes = [ctypes.POINTER(ctypes.c_float), i32]
     for fn in ("tlq_token_importance", "tlq_scale_candidates", "tlq_scale_candidates_noalloc", "tlq_quantize_weights", "tlq_pack_codes4", "tlq_quantize_activations", "tlq_scale_search_layer",
@@ -302,6 +304,15 @@ def tlq_debug_tile_walk(mtiles: int, otiles: int, K: int, n0: int, n1: int = 0, 
     visits = np.zeros((K, otiles, mtiles), dtype=np.int32)
     _check(lib.tlq_debug_tile_walk(mtiles, otiles, K, n0, n1, 1 if blocked else 0, block_a,
                                    visits.ctypes.data_as(ctypes.c_void_p)), "tlq_debug_tile_walk")
+    return visits
+
+
+def tlq_debug_resident_walk(mtiles: int, otiles: int, K: int, grid: int, blocked: bool = True):
+    """Host-side replay of the tile-resident kernels' work items -> numpy int32 [K, otiles, mtiles] of visit counts."""
+    import numpy as np
+    visits = np.zeros((K, otiles, mtiles), dtype=np.int32)
+    _check(lib.tlq_debug_resident_walk(mtiles, otiles, K, grid, 1 if blocked else 0,
+                                       visits.ctypes.data_as(ctypes.c_void_p)), "tlq_debug_resident_walk")
     return visits
 
 

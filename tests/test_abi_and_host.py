@@ -153,3 +153,14 @@ def test_tile_walk_visits_every_tile_exactly_once(tlq):
     assert tlq.lib.tlq_debug_tile_walk(4, 4, 1, 10, 138, 0, 8, args) == tlq.ERR_UNSUPPORTED
     assert tlq.lib.tlq_debug_tile_walk(4, 4, 0, 72, 76, 0, 8, args) == tlq.ERR_SHAPE
     assert tlq.lib.tlq_debug_tile_walk(4, 4, 1, 72, 76, 0, 8, None) == tlq.ERR_INVALID_ARG
+
+
+def test_resident_kernel_work_items_cover_every_candidate_of_every_tile_once(tlq):
+    """The tile-resident kernels: whole waves of tiles keep all K candidates, the tiles of the last partial wave are
+    split by candidates over the CTAs that would idle; with more CTAs than tiles everything is a tail."""
+    import numpy as np
+    for mtiles, otiles, K in ((64, 14, 20), (64, 2, 20), (64, 74, 20), (1, 1, 1), (3, 5, 7), (128, 6, 64), (33, 1, 2)):
+        for grid in (148, 132, 7, 1):
+            for blocked in (False, True):
+                v = tlq.tlq_debug_resident_walk(mtiles, otiles, K, min(grid, mtiles * otiles), blocked)
+                assert v.min() == 1 and v.max() == 1, (mtiles, otiles, K, grid, blocked)
