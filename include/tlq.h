@@ -245,6 +245,16 @@ int tlq_read_status(const void* workspace, void* stream);
 int tlq_selftest_bounded_wait(void* workspace, size_t workspace_bytes, int64_t limit_cycles, void* stream);
 
 /*
+ * Diagnostic (the paper has no counterpart): what the library measured about the current device's L2.  The L2 of this
+ * GPU is two partitions; the first large group-mode search on a device measures which partition each SM sits next to,
+ * and the fused bf16 GEMM then keeps each partition's CTAs to their own token tiles.  This call synchronises the device
+ * and copies the table to the HOST: info[0] = 1 if a usable table exists (0: not measured yet, or the measurement did
+ * not split the SMs into two clear groups, in which case the GEMM uses its plain tile order), info[1] = SMs measured,
+ * info[2], info[3] = SMs per partition; part (256 bytes, or NULL) = partition of each SM id.
+ */
+int tlq_l2_partition_info(int32_t* info /* host [4] */, uint8_t* part /* host [256] or NULL */);
+
+/*
  * Diagnostic, host only (the paper has no counterpart; no device is touched): the order in which the persistent CTAs
  * of the fused bf16 GEMM visit the (candidate, output tile, token tile) space, replayed on the host.  With n1 = 0
  * it is the walk of a grid of n0 CTAs (blocked != 0: by blocks of block_a token tiles); with n1 > 0 the walk of

@@ -182,7 +182,7 @@ const char* tlq_status_string(int status) {
   }
 }
 
-int tlq_version(void) { return 1006; }   // 1.6: bounded-wait self-test, tile-walk check
+int tlq_version(void) { return 1007; }   // 1.7: bounded-wait self-test, tile-walk checks, L2 partition table read-back
 
 int64_t tlq_kernel_launch_count(void) { return (int64_t)g_launch_count; }
 
@@ -494,6 +494,17 @@ int tlq_selftest_bounded_wait(void* workspace, size_t workspace_bytes, int64_t l
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   TLQ_CUDA_TRY(cudaMemsetAsync(workspace, 0, sizeof(WorkspaceHeader), st));
   return launch_bounded_wait_selftest(reinterpret_cast<WorkspaceHeader*>(workspace), (long long)limit_cycles, st);
+}
+
+int tlq_l2_partition_info(int32_t* info, uint8_t* part) {
+  if (info == nullptr) return TLQ_ERR_INVALID_ARG;
+  int rc = have_device();
+  if (rc != TLQ_OK) return rc;
+  L2PartMap m;
+  if ((rc = l2_partition_read(&m)) != TLQ_OK) return rc;
+  info[0] = m.valid; info[1] = m.n_sms; info[2] = m.count[0]; info[3] = m.count[1];
+  if (part != nullptr) memcpy(part, m.part, sizeof(m.part));
+  return TLQ_OK;
 }
 
 int tlq_debug_tile_walk(int64_t mtiles, int64_t otiles, int32_t K, int32_t n0, int32_t n1, int32_t blocked,

@@ -143,4 +143,14 @@ const L2PartMap* l2_partition_map(void* scratch, size_t scratch_bytes, cudaStrea
   return address[dev];
 }
 
+// Host copy of the current device's table (synchronises the device); TLQ_ERR_CUDA on failure.
+int l2_partition_read(L2PartMap* out) {
+  if (cudaDeviceSynchronize() != cudaSuccess) return TLQ_ERR_CUDA;
+  if (cudaMemcpyFromSymbol(out, g_l2_part_map, sizeof(L2PartMap)) != cudaSuccess) {
+    cudaGetLastError();
+    return TLQ_ERR_CUDA;
+  }
+  return TLQ_OK;
+}
+
 }  // namespace tlq

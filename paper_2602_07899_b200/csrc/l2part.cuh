@@ -30,6 +30,7 @@ struct L2PartMap {
 // A table that has not been measured yet has valid == 0.
 size_t l2_partition_scratch_bytes();
 const L2PartMap* l2_partition_map(void* scratch, size_t scratch_bytes, cudaStream_t st);
+int l2_partition_read(L2PartMap* out);      // host copy of the current device's table (synchronises the device)
 
 // This CTA's share of a (candidate, output tile, token tile) space.
 //

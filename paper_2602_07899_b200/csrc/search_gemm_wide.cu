@@ -271,8 +271,8 @@ int launch_search_gemm_bf16_wide(const uint16_t* X, const uint16_t* dW, const fl
   const int64_t tiles = (int64_t)plan.K * a.otiles * a.mpairs;
   const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
   // The partition-aware walk needs one CTA on every SM and enough tiles for the split to balance.  It is for
-  // activations that can stay in L2 (measured on the 7B-class layer: HBM bytes of the q / k / gate launches 1677 /
-  // 318 / 9700 MB -> 644 / 132 / 5240 MB); where they cannot, splitting the tokens only shortens the weight block a
+  // activations that can stay in L2 (measured on the 7B-class layer: HBM bytes of the q / k / gate launches about 1690 /
+  // 340 / 10460 MB -> 576 / 133 / 2813 MB, i.e. the operands once); where they cannot, splitting the tokens only shortens the weight block a
   // wave shares (18944-channel down-projection: 24.5 -> 45 GB), so the blocked walk stays whole.
   a.l2map = (grid == (unsigned)sms && tiles >= 8 * (int64_t)sms && !a.blocked) ? l2map : nullptr;
   gemm_bf16_wide_kernel<<<grid, kThreads, kSmemBytes, st>>>(tmA, tmB, a);

@@ -31,7 +31,7 @@ EXPORTS = (
     "tlq_status_string", "tlq_version", "tlq_token_importance", "tlq_scale_candidates_workspace_bytes",
     "tlq_scale_candidates", "tlq_scale_candidates_noalloc", "tlq_quantize_weights", "tlq_pack_codes4", "tlq_quantize_activations", "tlq_scale_search_workspace_bytes", "tlq_scale_search_layer", "tlq_scale_search_layer_two_stream",
     "tlq_apply_layer_workspace_bytes", "tlq_apply_layer", "tlq_read_status", "tlq_stage_timing_enable",
-    "tlq_stage_timing_drain", "tlq_kernel_launch_count", "tlq_selftest_bounded_wait", "tlq_debug_tile_walk", "tlq_debug_resident_walk",
+    "tlq_stage_timing_drain", "tlq_kernel_launch_count", "tlq_selftest_bounded_wait", "tlq_debug_tile_walk", "tlq_debug_resident_walk", "tlq_l2_partition_info",
 )
 
 
@@ -96,6 +96,8 @@ def _load() -> ctypes.CDLL:
     lib.tlq_selftest_bounded_wait.restype = i32
     lib.tlq_debug_tile_walk.argtypes = [i64, i64, i32, i32, i32, i32, i32, vp]
     lib.tlq_debug_tile_walk.restype = i32
+    lib.tlq_l2_partition_info.argtypes = [vp, vp]
+    lib.tlq_l2_partition_info.restype = i32
     lib.tlq_debug_resident_walk.argtypes = [i64, i64, i32, i32, i32, vp]
     lib.tlq_debug_resident_walk.restype = i32
     lib.tlq_stage_timing_enable.argtypes = [i32]
@@ -296,6 +298,15 @@ def tlq_selftest_bounded_wait(workspace: torch.Tensor, limit_cycles: int = 2_000
     _check(lib.tlq_selftest_bounded_wait(_ptr(workspace), workspace.numel() * workspace.element_size(), int(limit_cycles), st),
            "tlq_selftest_bounded_wait")
     return int(lib.tlq_read_status(_ptr(workspace), st))
+
+
+def tlq_l2_partition_info():
+    """-> dict(valid, n_sms, count=(n0, n1), part=numpy uint8 [256]): the current device's SM -> L2 partition table."""
+    import numpy as np
+    info = (ctypes.c_int32 * 4)()
+    part = np.zeros(256, dtype=np.uint8)
+    _check(lib.tlq_l2_partition_info(info, part.ctypes.data_as(ctypes.c_void_p)), "tlq_l2_partition_info")
+    return dict(valid=bool(info[0]), n_sms=int(info[1]), count=(int(info[2]), int(info[3])), part=part)
 
 
 def tlq_debug_tile_walk(mtiles: int, otiles: int, K: int, n0: int, n1: int = 0, blocked: bool = False, block_a: int = 8):

@@ -31,7 +31,7 @@ def test_every_declared_symbol_is_exported(tlq):
     for n in names:
         assert hasattr(tlq.lib, n), n
     assert sorted(tlq.EXPORTS) == names
-    assert tlq.lib.tlq_version() == 1006
+    assert tlq.lib.tlq_version() == 1007
     assert tlq.status_string(0) == "ok" and "workspace" in tlq.status_string(tlq.ERR_WORKSPACE)
 
 

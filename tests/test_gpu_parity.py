@@ -743,6 +743,13 @@ def test_search_with_the_l2_partition_aware_tile_walk(tlq, n, c2):
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     assert hdr[0] == 0 and int(hdr[5]) + int(hdr[6]) in (0, sms), hdr[:8]
     print("tile-walk slots claimed per L2 partition:", int(hdr[5]), int(hdr[6]))
+    info = tlq.tlq_l2_partition_info()
+    if info["valid"]:      # the walk used the table: as many slots per partition as the table has SMs
+        assert info["n_sms"] == sms and sum(info["count"]) == sms and min(info["count"]) * 4 >= sms
+        assert (int(hdr[5]), int(hdr[6])) == info["count"]
+        assert int(info["part"][:].max()) == 1
+    else:
+        assert int(hdr[5]) + int(hdr[6]) == 0
     # token skipping on top: the live token count, and with it the split, is only known on the device
     imp2 = imp.copy()
     imp2[np.random.default_rng(3).random(n) < 0.4] = 0.0
