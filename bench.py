@@ -526,6 +526,9 @@ def run_ours(args, cfgw):
                "kind": "oracle", "sample": sample_description(cfgw, BASELINE_TOKENS, BASELINE_LINEAR), "sample_seconds": round(dt, 3),
                "oracle_gflops": round(fl / dt / 1e9, 1)}
 
+    part = tlq.tlq_l2_partition_info()       # whether the bf16 GEMM ran its L2-partition-aware tile order on this device
+    l2_partitions = {"measured": part["valid"], "sms_per_partition": list(part["count"])}
+
     notes = (("" if args.linears is None else f" [subset: {args.linears}]")
              + ("" if args.importance == "config" else f" [importance: {args.importance}]")
              + (" [zero-weight tokens skipped]" if args.skip_zero_weight else "")
@@ -539,7 +542,7 @@ def run_ours(args, cfgw):
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": ms_e2e / args.steps},
             "gpu_launches": leg["launches"], "clocks": leg["clocks"], "per_linear": lin_report, "other_path_steps": extra,
-            "streaming_stages": streaming, "int8": int8_record}
+            "streaming_stages": streaming, "l2_partitions": l2_partitions, "int8": int8_record}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -89,6 +89,20 @@ extern "C" {
                                                stages the weight tile once for two 128-token halves (measured 8 %
                                                faster inside a benchmark step). */
 
+#define TLQ_FLAG_NO_REFINE 8u                /* tlq_scale_search_layer, group mode: skip the refine pass.  By default,
+                                               when other candidates' losses come within 1e-4 (relative) of the
+                                               smallest, those candidates (if there are no more than four, and no
+                                               more than K/2, of them: a flatter loss curve keeps its first result)
+                                               are evaluated a second time with delta weights split into two bf16
+                                               parts and short tensor-core accumulation chunks summed in registers
+                                               and fp64, which brings their losses from about 6e-5 to about 1e-6 of
+                                               the exact value; losses[] of those candidates, best_idx and s_best
+                                               come from the second evaluation.  per_token_err keeps the first
+                                               evaluation's values.  The pass costs a few idle launches when no
+                                               candidate is that close, and about four screening-candidates' time per
+                                               re-evaluated candidate when some are.  Not run by the two-stream call
+                                               nor in the symmetric modes (whose integer accumulation is exact). */
+
 #define TLQ_MAX_GRID 64
 
 typedef struct {

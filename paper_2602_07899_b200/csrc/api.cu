@@ -29,7 +29,8 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 int check_cfg(const tlq_config* cfg, int64_t C1, bool need_quantizer = true) {
   if (cfg == nullptr || cfg->struct_size != sizeof(tlq_config)) return TLQ_ERR_INVALID_ARG;
-  if ((cfg->flags & ~(uint32_t)(TLQ_FLAG_SKIP_ZERO_WEIGHT_TOKENS | TLQ_FLAG_GEMM_CTA_PAIRS | TLQ_FLAG_GEMM_NARROW_TILES)) != 0)
+  if ((cfg->flags & ~(uint32_t)(TLQ_FLAG_SKIP_ZERO_WEIGHT_TOKENS | TLQ_FLAG_GEMM_CTA_PAIRS | TLQ_FLAG_GEMM_NARROW_TILES |
+                                 TLQ_FLAG_NO_REFINE)) != 0)
     return TLQ_ERR_INVALID_ARG;
   if (cfg->n_grid < 1 || cfg->n_grid > TLQ_MAX_GRID) return TLQ_ERR_SHAPE;
   if (cfg->stat_mode < TLQ_STAT_MEAN_ABS || cfg->stat_mode > TLQ_STAT_MASKED_MAX) return TLQ_ERR_INVALID_ARG;
@@ -89,6 +90,8 @@ struct SearchLayout {
   int32_t* live_idx;     // [N] source row of each packed row
   float* wc;             // [n_pad] packed weights
   uint16_t* Xc;          // [n_pad, C1] packed activations
+  double* refine_partials; // group mode: [kMaxRefine][refine_per_r] weighted tile sums of the refine pass
+  int64_t refine_per_r;
   size_t bytes;
   GemmPlan plan;         // the mode's own GEMM
   GemmPlan plan_resident; // the tile-resident kernel's (all candidates per tile): symmetric modes and the two-stream search
@@ -112,6 +115,8 @@ SearchLayout carve_search(void* ws, int64_t N, int64_t C1, int64_t C2, const tlq
   L.ptab = c.take<float>((size_t)K * L.ptab_slices * L.plan.n_pad);
   if (cfg->mode == TLQ_W4A16_ASYM_GROUP) {
     L.dW = c.take<uint16_t>((size_t)K * C2 * C1, 1024);
+    L.refine_per_r = refine_partials_per_candidate(N, C2);
+    L.refine_partials = c.take<double>((size_t)kMaxRefine * L.refine_per_r);
   } else {
     L.Wq = c.take<int8_t>((size_t)K * C2 * C1, 1024);
     L.u = c.take<float>((size_t)K * C2);
@@ -182,7 +187,7 @@ const char* tlq_status_string(int status) {
   }
 }
 
-int tlq_version(void) { return 1007; }   // 1.7: bounded-wait self-test, tile-walk checks, L2 partition table read-back
+int tlq_version(void) { return 1008; }   // 1.8: refine pass of the group-mode search (TLQ_FLAG_NO_REFINE)
 
 int64_t tlq_kernel_launch_count(void) { return (int64_t)g_launch_count; }
 
@@ -381,6 +386,20 @@ static int search_impl(const void* X, const void* X_ref, int64_t N, int64_t C1, 
   if ((rc = launch_loss_reduce(L.partials, used.partials_per_k, K, w_imp, N, C2, L.s, C1, L.hdr, losses, best_idx,
                                reinterpret_cast<uint16_t*>(s_best), st)) != TLQ_OK)
     return rc;
+  // Candidates too close to the minimum for the screening arithmetic to order are evaluated again, more exactly; the
+  // set is chosen on the device, so the kernels are enqueued regardless and return at once when it is empty.
+  if (cfg->mode == TLQ_W4A16_ASYM_GROUP && !two_stream && K >= 2 && (cfg->flags & TLQ_FLAG_NO_REFINE) == 0) {
+    TLQ_CUDA_TRY(cudaMemsetAsync(L.refine_partials, 0, (size_t)kMaxRefine * L.refine_per_r * sizeof(double), st));
+    if ((rc = launch_refine_select(losses, K, L.hdr, st)) != TLQ_OK) return rc;
+    if ((rc = launch_fakequant_group_residual(Wb, L.s, L.rs, C2, C1, cfg->group_size, cfg->w_bits, L.dW, L.hdr, st)) !=
+        TLQ_OK)
+      return rc;
+    if ((rc = launch_search_gemm_refine(Xg, L.dW, wg, N, C1, C2, K, L.refine_partials, L.hdr, n_live, st)) != TLQ_OK)
+      return rc;
+    if ((rc = launch_refine_finish(L.refine_partials, L.refine_per_r, L.s, C1, L.hdr, losses, best_idx,
+                                   reinterpret_cast<uint16_t*>(s_best), st)) != TLQ_OK)
+      return rc;
+  }
   if (per_token_err != nullptr)
     if ((rc = launch_per_token_reduce(L.ptab, K, used.otiles * (resident ? 2 : 1), used.n_pad, N, per_token_err, st)) != TLQ_OK)
       return rc;

@@ -168,6 +168,7 @@ __host__ __device__ inline bool work_item(const TailSplit& t, int w, int K, int&
 // ---------------------------------------------------------------------------------------------
 // Workspace header (first 256 bytes of every workspace)
 // ---------------------------------------------------------------------------------------------
+constexpr int kMaxRefine = 4;            // candidates the refine pass re-evaluates at most
 struct WorkspaceHeader {
   int32_t status;     // TLQ_OK / TLQ_ERR_TIMEOUT / TLQ_ERR_NONFINITE
   int32_t where;      // diagnostic: which wait gave up
@@ -175,7 +176,16 @@ struct WorkspaceHeader {
   int32_t reduce_done; // CTAs of the loss reduction that have finished (the header is zeroed by every call)
   int32_t selftest;    // set by the bounded-wait self-test when its abort flag reached the other lanes
   int32_t slot_count[2]; // tile-walk slots claimed so far in each L2 partition by the CTAs of the search GEMM
-  int32_t pad[57];
+  // refine pass (reduce.cu, search_refine.cu): the candidates whose screened losses lie within the band of the
+  // minimum, lowest loss first, and for each the slot of the delta-weight buffer (a candidate outside the list, whose
+  // delta weights are no longer needed) that receives the low part of its split delta weights
+  int32_t refine_count;
+  int32_t refine_cand[kMaxRefine];
+  int32_t refine_slot[kMaxRefine];
+  int32_t refine_done;   // CTAs of the refine reduction that have finished
+  int32_t pad0;
+  double denom;          // C2 * sum of the token weights: what the weighted partial sums are divided by
+  int32_t pad[44];
 };
 static_assert(sizeof(WorkspaceHeader) == 256, "header is 256 bytes");
 
@@ -227,6 +237,28 @@ int launch_loss_reduce(const float* partials, int64_t per_k, int K, const float*
                        uint16_t* s_best, cudaStream_t st);
 int launch_per_token_reduce(const float* ptab /*[K,otiles,Npad]*/, int K, int64_t otiles, int64_t Npad, int64_t N,
                             float* per_token /*[K,N]*/, cudaStream_t st);
+
+// Refine pass of the group-mode search (16-bit activations).  The screening GEMM sees delta weights rounded to bf16
+// and accumulates each output over all of C1 in the tensor core's fp32 accumulator, which shifts a loss by up to
+// 6e-5 relative; when two candidates are closer than that, the candidates within kRefineBand of the minimum are
+// evaluated again with split delta weights (bf16 high + bf16 low part) and short accumulation chunks summed outside
+// the tensor core, and the argmin is taken on those values.
+constexpr double kRefineBand = 1.0e-4;
+// reduce.cu: picks the refine set into hdr: 2 .. min(kMaxRefine, K/2) candidates, or none
+int launch_refine_select(const double* losses, int K, WorkspaceHeader* hdr, cudaStream_t st);
+// reduce.cu: refined losses from the fp64 partials [kMaxRefine][per_r]; rewrites losses[k] of the refined
+// candidates, the argmin and the winning scale row
+int launch_refine_finish(const double* partials, int64_t per_r, const uint16_t* s_table, int64_t C1,
+                         WorkspaceHeader* hdr, double* losses, int32_t* best_idx, uint16_t* s_best, cudaStream_t st);
+// fakequant.cu: for each refined candidate r, bf16(dW - bf16(dW)) of candidate hdr->refine_cand[r] into slot
+// hdr->refine_slot[r] of dW [K,C2,C1]
+int launch_fakequant_group_residual(const uint16_t* W, const uint16_t* s, const float* rs, int64_t C2, int64_t C1,
+                                    int group, int w_bits, uint16_t* dW, const WorkspaceHeader* hdr, cudaStream_t st);
+// search_refine.cu: partials [kMaxRefine][refine_partials_per_candidate] (fp64, zeroed by the caller)
+int64_t refine_partials_per_candidate(int64_t N, int64_t C2);
+int launch_search_gemm_refine(const uint16_t* X, const uint16_t* dW, const float* w_imp, int64_t N, int64_t C1,
+                              int64_t C2, int K, double* partials, WorkspaceHeader* hdr, const int32_t* n_live,
+                              cudaStream_t st);
 
 // selftest.cu: one warp waits `limit_cycles` on a barrier nobody arrives on, then reports TLQ_ERR_TIMEOUT in `hdr`
 int launch_bounded_wait_selftest(WorkspaceHeader* hdr, long long limit_cycles, cudaStream_t st);

@@ -307,8 +307,11 @@ __global__ void __launch_bounds__(kGqThreads)
 fakequant_group_kernel(const uint16_t* __restrict__ W, const uint16_t* __restrict__ s_tab,
                        const float* __restrict__ rs_tab, int K, int k_per_cta, int64_t C2, int64_t C1, int group,
                        int qmax, uint16_t* __restrict__ dW, uint8_t* __restrict__ codes, float* __restrict__ steps,
-                       int32_t* __restrict__ zeros) {
+                       int32_t* __restrict__ zeros, const WorkspaceHeader* __restrict__ refine) {
   __shared__ uint4 tile[kGqRows][kGqCols / 8];
+  // Residual mode (refine pass of the search): blockIdx.y names an entry of the refine set; the candidate's delta
+  // weights d are formed as always and what is stored, in the slot the set assigns, is bf16(d - bf16(d)).
+  if (refine != nullptr && (int)blockIdx.y >= refine->refine_count) return;
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const int64_t col_blocks = (C1 + kGqCols - 1) / kGqCols;      // grid.x = column blocks x row tiles, columns fastest
@@ -318,8 +321,9 @@ fakequant_group_kernel(const uint16_t* __restrict__ W, const uint16_t* __restric
   const int lanes_per_group = group >> 4;
   const float qmax_f = (float)qmax;
   const int64_t ngroups = C1 / group;
-  const int k_begin = blockIdx.y * k_per_cta;
-  const int k_end = min(K, k_begin + k_per_cta);
+  const int k_begin = refine != nullptr ? refine->refine_cand[blockIdx.y] : blockIdx.y * k_per_cta;
+  const int k_end = refine != nullptr ? k_begin + 1 : min(K, k_begin + k_per_cta);
+  const int k_shift = refine != nullptr ? refine->refine_slot[blockIdx.y] - k_begin : 0;   // output slot - candidate
 
   // stage the W tile (zeros outside the matrix)
 #pragma unroll
@@ -403,11 +407,16 @@ fakequant_group_kernel(const uint16_t* __restrict__ W, const uint16_t* __restric
             qpack[(j + h) >> 2] |= (__float_as_uint(__fadd_rn(__fadd_rn(qz, zf), kMagic)) & 0xFFu) << (((j + h) & 3) * 8);
         }
         outw[j >> 1] = pack_bf16x2(d[0], d[1]);
+        if (refine != nullptr) {      // d - bf16(d) is exact in binary32; its own bf16 rounding leaves 2^-18 |d|
+          const uint32_t hi = outw[j >> 1];
+          outw[j >> 1] = pack_bf16x2(__fsub_rn(d[0], __uint_as_float(hi << 16)),
+                                     __fsub_rn(d[1], __uint_as_float(hi & 0xFFFF0000u)));
+        }
       }
       const int64_t row = row0 + r;
       if (col_ok && row < C2) {
         if (dW != nullptr) {
-          uint4* dst = reinterpret_cast<uint4*>(dW + ((int64_t)k * C2 + row) * C1 + c0);
+          uint4* dst = reinterpret_cast<uint4*>(dW + ((int64_t)(k + k_shift) * C2 + row) * C1 + c0);
           dst[0] = make_uint4(outw[0], outw[1], outw[2], outw[3]);
           dst[1] = make_uint4(outw[4], outw[5], outw[6], outw[7]);
         }
@@ -451,7 +460,15 @@ int launch_fakequant_group(const uint16_t* W, const uint16_t* s, const float* rs
     return after_launch();
   }
   fakequant_group_kernel<<<grid, kGqThreads, 0, st>>>(W, s, rs, K, k_per_cta, C2, C1, group, (1 << w_bits) - 1, dW,
-                                                     codes, steps, zeros);
+                                                     codes, steps, zeros, nullptr);
+  return after_launch();
+}
+
+int launch_fakequant_group_residual(const uint16_t* W, const uint16_t* s, const float* rs, int64_t C2, int64_t C1,
+                                    int group, int w_bits, uint16_t* dW, const WorkspaceHeader* hdr, cudaStream_t st) {
+  dim3 grid((unsigned)(ceil_div(C1, kGqCols) * ceil_div(C2, kGqRows)), (unsigned)kMaxRefine);
+  fakequant_group_kernel<<<grid, kGqThreads, 0, st>>>(W, s, rs, 0, 1, C2, C1, group, (1 << w_bits) - 1, dW, nullptr,
+                                                     nullptr, nullptr, hdr);
   return after_launch();
 }
 

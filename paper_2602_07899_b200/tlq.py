@@ -50,6 +50,7 @@ class Config(ctypes.Structure):
 FLAG_SKIP_ZERO_WEIGHT_TOKENS = 1
 FLAG_GEMM_CTA_PAIRS = 2
 FLAG_GEMM_NARROW_TILES = 4
+FLAG_NO_REFINE = 8
 
 
 def config(mode: int = W4A16_ASYM_GROUP, w_bits: Optional[int] = None, a_bits: Optional[int] = None,

@@ -31,7 +31,7 @@ def test_every_declared_symbol_is_exported(tlq):
     for n in names:
         assert hasattr(tlq.lib, n), n
     assert sorted(tlq.EXPORTS) == names
-    assert tlq.lib.tlq_version() == 1007
+    assert tlq.lib.tlq_version() == 1008
     assert tlq.status_string(0) == "ok" and "workspace" in tlq.status_string(tlq.ERR_WORKSPACE)
 
 
@@ -91,7 +91,7 @@ def test_host_validation_error_codes(tlq):
     assert L.tlq_scale_search_layer(a, 4, 128, a, 8, None, None, ctypes.byref(cm), a, 1 << 30, a, a, a, None,
                                     None) == tlq.ERR_INVALID_ARG
     # flags: unknown bits, token skipping without weights or with a per-token table, options the two-stream call rejects
-    assert L.tlq_scale_search_layer(a, 4, 128, a, 8, None, None, ctypes.byref(tlq.config(flags=8)), a, 1 << 30, a, a, a,
+    assert L.tlq_scale_search_layer(a, 4, 128, a, 8, None, None, ctypes.byref(tlq.config(flags=16)), a, 1 << 30, a, a, a,
                                     None, None) == tlq.ERR_INVALID_ARG
     skip = tlq.config(flags=tlq.FLAG_SKIP_ZERO_WEIGHT_TOKENS)
     assert L.tlq_scale_search_layer(a, 4, 128, a, 8, None, None, ctypes.byref(skip), a, 1 << 30, a, a, a, None,
