@@ -414,6 +414,8 @@ def run_ours(args, cfgw):
 
     flags = tlq.FLAG_SKIP_ZERO_WEIGHT_TOKENS if args.skip_zero_weight else 0
     flags |= {"default": 0, "pairs": tlq.FLAG_GEMM_CTA_PAIRS, "narrow": tlq.FLAG_GEMM_NARROW_TILES}[args.gemm]
+    if args.no_refine:
+        flags |= tlq.FLAG_NO_REFINE
     cfg = search_config(tlq, cfgr, flags)
 
     # host (pinned) copies for the end-to-end leg, device-resident copies for the kernel leg
@@ -444,7 +446,7 @@ def run_ours(args, cfgw):
     #      applying the winner (Y_q for the next layer) and the token-importance reduction
     extra = side_legs(tlq, torch, dev, cfgr, cfg, lins, dev_x, dev_w, leg["bufs"], peaks)
     plain = (args.linears is None and args.mode is None and not args.skip_zero_weight and args.gemm == "default"
-             and not args.shared_scale and args.importance == "config")
+             and not args.shared_scale and args.importance == "config" and not args.no_refine)
     del leg["bufs"], leg["workspace"]
     torch.cuda.empty_cache()
 
@@ -532,6 +534,7 @@ def run_ours(args, cfgw):
     notes = (("" if args.linears is None else f" [subset: {args.linears}]")
              + ("" if args.importance == "config" else f" [importance: {args.importance}]")
              + (" [zero-weight tokens skipped]" if args.skip_zero_weight else "")
+             + (" [refine pass off]" if args.no_refine else "")
              + (" [shared scale: " + ", ".join(l.name for l in lins) + "]" if args.shared_scale else ""))
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak",
@@ -566,6 +569,8 @@ def main():
                     help="stack linears that share their input (q/k/v, gate/up) and search one scale for each stack")
     ap.add_argument("--linears", default=None, help="comma-separated subset of q,k,v,o,gate,up,down (profiling)")
     ap.add_argument("--profile", action="store_true", help="kernel leg only: skip the end-to-end and CPU legs")
+    ap.add_argument("--no-refine", action="store_true",
+                    help="set TLQ_FLAG_NO_REFINE (the second evaluation of near-tied candidates), for A/B measurements")
     ap.add_argument("--no-int8", action="store_true", help="skip the W8A8 sub-record of the default (cfg1) run")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

@@ -383,14 +383,16 @@ static int search_impl(const void* X, const void* X_ref, int64_t N, int64_t C1, 
   if ((rc = timing_mark(3, st)) != TLQ_OK) return rc;
   const bool resident = two_stream || cfg->mode != TLQ_W4A16_ASYM_GROUP;
   const GemmPlan& used = resident ? L.plan_resident : L.plan;
+  const bool refine =
+      cfg->mode == TLQ_W4A16_ASYM_GROUP && !two_stream && K >= 2 && (cfg->flags & TLQ_FLAG_NO_REFINE) == 0;
   if ((rc = launch_loss_reduce(L.partials, used.partials_per_k, K, w_imp, N, C2, L.s, C1, L.hdr, losses, best_idx,
-                               reinterpret_cast<uint16_t*>(s_best), st)) != TLQ_OK)
+                               reinterpret_cast<uint16_t*>(s_best), refine, st)) != TLQ_OK)
     return rc;
   // Candidates too close to the minimum for the screening arithmetic to order are evaluated again, more exactly; the
   // set is chosen on the device, so the kernels are enqueued regardless and return at once when it is empty.
-  if (cfg->mode == TLQ_W4A16_ASYM_GROUP && !two_stream && K >= 2 && (cfg->flags & TLQ_FLAG_NO_REFINE) == 0) {
-    TLQ_CUDA_TRY(cudaMemsetAsync(L.refine_partials, 0, (size_t)kMaxRefine * L.refine_per_r * sizeof(double), st));
-    if ((rc = launch_refine_select(losses, K, L.hdr, st)) != TLQ_OK) return rc;
+  if (refine) {
+    if (compact)      // token tiles without live tokens are not visited
+      TLQ_CUDA_TRY(cudaMemsetAsync(L.refine_partials, 0, (size_t)kMaxRefine * L.refine_per_r * sizeof(double), st));
     if ((rc = launch_fakequant_group_residual(Wb, L.s, L.rs, C2, C1, cfg->group_size, cfg->w_bits, L.dW, L.hdr, st)) !=
         TLQ_OK)
       return rc;

@@ -234,7 +234,8 @@ int launch_top_mask(const float* imp, int64_t N, int64_t k_sel, uint8_t* mask, c
 // reduce.cu
 int launch_loss_reduce(const float* partials, int64_t per_k, int K, const float* w_imp, int64_t N, int64_t C2,
                        const uint16_t* s_table, int64_t C1, WorkspaceHeader* hdr, double* losses, int32_t* best_idx,
-                       uint16_t* s_best, cudaStream_t st);
+                       uint16_t* s_best, bool pick_refine_set /* also fill hdr's refine set: 2 .. min(kMaxRefine, K/2)
+                       candidates, or none */, cudaStream_t st);
 int launch_per_token_reduce(const float* ptab /*[K,otiles,Npad]*/, int K, int64_t otiles, int64_t Npad, int64_t N,
                             float* per_token /*[K,N]*/, cudaStream_t st);
 
@@ -244,8 +245,6 @@ int launch_per_token_reduce(const float* ptab /*[K,otiles,Npad]*/, int K, int64_
 // evaluated again with split delta weights (bf16 high + bf16 low part) and short accumulation chunks summed outside
 // the tensor core, and the argmin is taken on those values.
 constexpr double kRefineBand = 1.0e-4;
-// reduce.cu: picks the refine set into hdr: 2 .. min(kMaxRefine, K/2) candidates, or none
-int launch_refine_select(const double* losses, int K, WorkspaceHeader* hdr, cudaStream_t st);
 // reduce.cu: refined losses from the fp64 partials [kMaxRefine][per_r]; rewrites losses[k] of the refined
 // candidates, the argmin and the winning scale row
 int launch_refine_finish(const double* partials, int64_t per_r, const uint16_t* s_table, int64_t C1,
@@ -254,7 +253,8 @@ int launch_refine_finish(const double* partials, int64_t per_r, const uint16_t* 
 // hdr->refine_slot[r] of dW [K,C2,C1]
 int launch_fakequant_group_residual(const uint16_t* W, const uint16_t* s, const float* rs, int64_t C2, int64_t C1,
                                     int group, int w_bits, uint16_t* dW, const WorkspaceHeader* hdr, cudaStream_t st);
-// search_refine.cu: partials [kMaxRefine][refine_partials_per_candidate] (fp64, zeroed by the caller)
+// search_refine.cu: partials [kMaxRefine][refine_partials_per_candidate] (fp64; zeroed by the caller when n_live is
+// given, since token tiles without live tokens are not written)
 int64_t refine_partials_per_candidate(int64_t N, int64_t C2);
 int launch_search_gemm_refine(const uint16_t* X, const uint16_t* dW, const float* w_imp, int64_t N, int64_t C1,
                               int64_t C2, int K, double* partials, WorkspaceHeader* hdr, const int32_t* n_live,

@@ -307,16 +307,16 @@ __global__ void __launch_bounds__(kGqThreads)
 fakequant_group_kernel(const uint16_t* __restrict__ W, const uint16_t* __restrict__ s_tab,
                        const float* __restrict__ rs_tab, int K, int k_per_cta, int64_t C2, int64_t C1, int group,
                        int qmax, uint16_t* __restrict__ dW, uint8_t* __restrict__ codes, float* __restrict__ steps,
-                       int32_t* __restrict__ zeros, const WorkspaceHeader* __restrict__ refine) {
+                       int32_t* __restrict__ zeros, const WorkspaceHeader* __restrict__ refine, int row_tiles_per_cta) {
   __shared__ uint4 tile[kGqRows][kGqCols / 8];
   // Residual mode (refine pass of the search): blockIdx.y names an entry of the refine set; the candidate's delta
   // weights d are formed as always and what is stored, in the slot the set assigns, is bf16(d - bf16(d)).
   if (refine != nullptr && (int)blockIdx.y >= refine->refine_count) return;
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
-  const int64_t col_blocks = (C1 + kGqCols - 1) / kGqCols;      // grid.x = column blocks x row tiles, columns fastest
+  const int64_t col_blocks = (C1 + kGqCols - 1) / kGqCols;      // grid.x = column blocks x runs of row tiles
   const int64_t c0 = (int64_t)(blockIdx.x % col_blocks) * kGqCols + lane * 16;
-  const int64_t row0 = (int64_t)(blockIdx.x / col_blocks) * kGqRows;
+  const int64_t row_tile0 = (int64_t)(blockIdx.x / col_blocks) * row_tiles_per_cta;
   const bool col_ok = c0 < C1;                    // C1 % 16 == 0 is guaranteed by the group sizes
   const int lanes_per_group = group >> 4;
   const float qmax_f = (float)qmax;
@@ -325,107 +325,112 @@ fakequant_group_kernel(const uint16_t* __restrict__ W, const uint16_t* __restric
   const int k_end = refine != nullptr ? k_begin + 1 : min(K, k_begin + k_per_cta);
   const int k_shift = refine != nullptr ? refine->refine_slot[blockIdx.y] - k_begin : 0;   // output slot - candidate
 
-  // stage the W tile (zeros outside the matrix)
+  for (int rt = 0; rt < row_tiles_per_cta; ++rt) {
+    const int64_t row0 = (row_tile0 + rt) * kGqRows;
+    if (row0 >= C2) break;
+    if (rt > 0) __syncthreads();                  // the previous tile has been read by every warp
+    // stage the W tile (zeros outside the matrix)
 #pragma unroll
-  for (int p = 0; p < kGqRows / 8; ++p) {
-    const int r = p * 8 + warp;
-    uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0;
-    if (col_ok && row0 + r < C2) {
-      const uint16_t* src = W + (row0 + r) * C1 + c0;
-      v0 = ld_nc_16(src);
-      v1 = ld_nc_16(src + 8);
+    for (int p = 0; p < kGqRows / 8; ++p) {
+      const int r = p * 8 + warp;
+      uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0;
+      if (col_ok && row0 + r < C2) {
+        const uint16_t* src = W + (row0 + r) * C1 + c0;
+        v0 = ld_nc_16(src);
+        v1 = ld_nc_16(src + 8);
+      }
+      tile[r][lane * 2] = v0;
+      tile[r][lane * 2 + 1] = v1;
     }
-    tile[r][lane * 2] = v0;
-    tile[r][lane * 2 + 1] = v1;
-  }
-  __syncthreads();
+    __syncthreads();
 
-  for (int k = k_begin; k < k_end; ++k) {
-    float sv[16], rsv[16];
-    if (s_tab != nullptr && col_ok) {
-      const uint16_t* sp = s_tab + (int64_t)k * C1 + c0;
-      float a[8], b[8];
-      unpack8(*reinterpret_cast<const uint4*>(sp), a);
-      unpack8(*reinterpret_cast<const uint4*>(sp + 8), b);
+    for (int k = k_begin; k < k_end; ++k) {
+      float sv[16], rsv[16];
+      if (s_tab != nullptr && col_ok) {
+        const uint16_t* sp = s_tab + (int64_t)k * C1 + c0;
+        float a[8], b[8];
+        unpack8(*reinterpret_cast<const uint4*>(sp), a);
+        unpack8(*reinterpret_cast<const uint4*>(sp + 8), b);
 #pragma unroll
-      for (int j = 0; j < 8; ++j) { sv[j] = a[j]; sv[8 + j] = b[j]; }
-      if (rs_tab != nullptr) {
-        const float4* rp = reinterpret_cast<const float4*>(rs_tab + (int64_t)k * C1 + c0);
+        for (int j = 0; j < 8; ++j) { sv[j] = a[j]; sv[8 + j] = b[j]; }
+        if (rs_tab != nullptr) {
+          const float4* rp = reinterpret_cast<const float4*>(rs_tab + (int64_t)k * C1 + c0);
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const float4 r4 = rp[j];
-          rsv[j * 4] = r4.x; rsv[j * 4 + 1] = r4.y; rsv[j * 4 + 2] = r4.z; rsv[j * 4 + 3] = r4.w;
+          for (int j = 0; j < 4; ++j) {
+            const float4 r4 = rp[j];
+            rsv[j * 4] = r4.x; rsv[j * 4 + 1] = r4.y; rsv[j * 4 + 2] = r4.z; rsv[j * 4 + 3] = r4.w;
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) rsv[j] = __fdiv_rn(1.0f, sv[j]);
         }
       } else {
 #pragma unroll
-        for (int j = 0; j < 16; ++j) rsv[j] = __fdiv_rn(1.0f, sv[j]);
+        for (int j = 0; j < 16; ++j) { sv[j] = 1.0f; rsv[j] = 1.0f; }
       }
-    } else {
-#pragma unroll
-      for (int j = 0; j < 16; ++j) { sv[j] = 1.0f; rsv[j] = 1.0f; }
-    }
 #pragma unroll 1
-    for (int p = 0; p < kGqRows / 8; ++p) {
-      const int r = p * 8 + warp;
-      float w[16], pr[16];
-      {
-        float a[8], b[8];
-        unpack8(tile[r][lane * 2], a);
-        unpack8(tile[r][lane * 2 + 1], b);
+      for (int p = 0; p < kGqRows / 8; ++p) {
+        const int r = p * 8 + warp;
+        float w[16], pr[16];
+        {
+          float a[8], b[8];
+          unpack8(tile[r][lane * 2], a);
+          unpack8(tile[r][lane * 2 + 1], b);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { w[j] = a[j]; w[8 + j] = b[j]; }
-      }
-      float mx, mn;
+          for (int j = 0; j < 8; ++j) { w[j] = a[j]; w[8 + j] = b[j]; }
+        }
+        float mx, mn;
 #pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        pr[j] = __fmul_rn(sv[j], w[j]);            // exact: 8-bit x 8-bit significands
-        mx = (j == 0) ? pr[0] : fmaxf(mx, pr[j]);
-        mn = (j == 0) ? pr[0] : fminf(mn, pr[j]);
-      }
-      for (int off = 1; off < lanes_per_group; off <<= 1) {
-        mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
-        mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, off));
-      }
-      const float range = fmaxf(__fsub_rn(mx, mn), TLQ_RANGE_FLOOR);
-      const float step = __fdiv_rn(range, qmax_f);
-      const float inv = rcp_fast(step);
-      // zero-point z = clamp(-rint(mn / step), 0, qmax), kept as a float
-      const float zf = -quotient_rint_clamped(mn, step, inv, -qmax_f, 0.0f);
-      const float lo = -zf, hi = qmax_f - zf;          // bounds of q - z
-      uint32_t outw[8];
-      uint32_t qpack[4] = {0u, 0u, 0u, 0u};
+        for (int j = 0; j < 16; ++j) {
+          pr[j] = __fmul_rn(sv[j], w[j]);            // exact: 8-bit x 8-bit significands
+          mx = (j == 0) ? pr[0] : fmaxf(mx, pr[j]);
+          mn = (j == 0) ? pr[0] : fminf(mn, pr[j]);
+        }
+        for (int off = 1; off < lanes_per_group; off <<= 1) {
+          mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
+          mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, off));
+        }
+        const float range = fmaxf(__fsub_rn(mx, mn), TLQ_RANGE_FLOOR);
+        const float step = __fdiv_rn(range, qmax_f);
+        const float inv = rcp_fast(step);
+        // zero-point z = clamp(-rint(mn / step), 0, qmax), kept as a float
+        const float zf = -quotient_rint_clamped(mn, step, inv, -qmax_f, 0.0f);
+        const float lo = -zf, hi = qmax_f - zf;          // bounds of q - z
+        uint32_t outw[8];
+        uint32_t qpack[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
-      for (int j = 0; j < 16; j += 2) {
-        float d[2];
+        for (int j = 0; j < 16; j += 2) {
+          float d[2];
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const float qz = quotient_rint_clamped(pr[j + h], step, inv, lo, hi);     // q - z
-          const float dq = __fmul_rn(qz, step);
-          const float w_hat = __fmul_rn(dq, rsv[j + h]);
-          d[h] = __fsub_rn(w[j + h], w_hat);
+          for (int h = 0; h < 2; ++h) {
+            const float qz = quotient_rint_clamped(pr[j + h], step, inv, lo, hi);     // q - z
+            const float dq = __fmul_rn(qz, step);
+            const float w_hat = __fmul_rn(dq, rsv[j + h]);
+            d[h] = __fsub_rn(w[j + h], w_hat);
+            if (codes != nullptr)
+              qpack[(j + h) >> 2] |= (__float_as_uint(__fadd_rn(__fadd_rn(qz, zf), kMagic)) & 0xFFu) << (((j + h) & 3) * 8);
+          }
+          outw[j >> 1] = pack_bf16x2(d[0], d[1]);
+          if (refine != nullptr) {      // d - bf16(d) is exact in binary32; its own bf16 rounding leaves 2^-18 |d|
+            const uint32_t hi = outw[j >> 1];
+            outw[j >> 1] = pack_bf16x2(__fsub_rn(d[0], __uint_as_float(hi << 16)),
+                                       __fsub_rn(d[1], __uint_as_float(hi & 0xFFFF0000u)));
+          }
+        }
+        const int64_t row = row0 + r;
+        if (col_ok && row < C2) {
+          if (dW != nullptr) {
+            uint4* dst = reinterpret_cast<uint4*>(dW + ((int64_t)(k + k_shift) * C2 + row) * C1 + c0);
+            dst[0] = make_uint4(outw[0], outw[1], outw[2], outw[3]);
+            dst[1] = make_uint4(outw[4], outw[5], outw[6], outw[7]);
+          }
           if (codes != nullptr)
-            qpack[(j + h) >> 2] |= (__float_as_uint(__fadd_rn(__fadd_rn(qz, zf), kMagic)) & 0xFFu) << (((j + h) & 3) * 8);
-        }
-        outw[j >> 1] = pack_bf16x2(d[0], d[1]);
-        if (refine != nullptr) {      // d - bf16(d) is exact in binary32; its own bf16 rounding leaves 2^-18 |d|
-          const uint32_t hi = outw[j >> 1];
-          outw[j >> 1] = pack_bf16x2(__fsub_rn(d[0], __uint_as_float(hi << 16)),
-                                     __fsub_rn(d[1], __uint_as_float(hi & 0xFFFF0000u)));
-        }
-      }
-      const int64_t row = row0 + r;
-      if (col_ok && row < C2) {
-        if (dW != nullptr) {
-          uint4* dst = reinterpret_cast<uint4*>(dW + ((int64_t)(k + k_shift) * C2 + row) * C1 + c0);
-          dst[0] = make_uint4(outw[0], outw[1], outw[2], outw[3]);
-          dst[1] = make_uint4(outw[4], outw[5], outw[6], outw[7]);
-        }
-        if (codes != nullptr)
-          *reinterpret_cast<uint4*>(codes + row * C1 + c0) = make_uint4(qpack[0], qpack[1], qpack[2], qpack[3]);
-        if ((lane % lanes_per_group) == 0) {
-          const int64_t g = c0 / group;
-          if (steps != nullptr) steps[row * ngroups + g] = step;
-          if (zeros != nullptr) zeros[row * ngroups + g] = (int)zf;
+            *reinterpret_cast<uint4*>(codes + row * C1 + c0) = make_uint4(qpack[0], qpack[1], qpack[2], qpack[3]);
+          if ((lane % lanes_per_group) == 0) {
+            const int64_t g = c0 / group;
+            if (steps != nullptr) steps[row * ngroups + g] = step;
+            if (zeros != nullptr) zeros[row * ngroups + g] = (int)zf;
+          }
         }
       }
     }
@@ -460,15 +465,17 @@ int launch_fakequant_group(const uint16_t* W, const uint16_t* s, const float* rs
     return after_launch();
   }
   fakequant_group_kernel<<<grid, kGqThreads, 0, st>>>(W, s, rs, K, k_per_cta, C2, C1, group, (1 << w_bits) - 1, dW,
-                                                     codes, steps, zeros, nullptr);
+                                                     codes, steps, zeros, nullptr, 1);
   return after_launch();
 }
 
 int launch_fakequant_group_residual(const uint16_t* W, const uint16_t* s, const float* rs, int64_t C2, int64_t C1,
                                     int group, int w_bits, uint16_t* dW, const WorkspaceHeader* hdr, cudaStream_t st) {
-  dim3 grid((unsigned)(ceil_div(C1, kGqCols) * ceil_div(C2, kGqRows)), (unsigned)kMaxRefine);
+  // launched whether or not there is a refine set: few CTAs, each walking a run of row tiles
+  constexpr int kRun = 8;
+  dim3 grid((unsigned)(ceil_div(C1, kGqCols) * ceil_div(ceil_div(C2, kGqRows), kRun)), (unsigned)kMaxRefine);
   fakequant_group_kernel<<<grid, kGqThreads, 0, st>>>(W, s, rs, 0, 1, C2, C1, group, (1 << w_bits) - 1, dW, nullptr,
-                                                     nullptr, nullptr, hdr);
+                                                     nullptr, nullptr, hdr, kRun);
   return after_launch();
 }
 

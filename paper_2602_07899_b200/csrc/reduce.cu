@@ -21,11 +21,52 @@ __device__ __forceinline__ double block_sum_fixed(double v, double* scratch) {
   return scratch[0];
 }
 
+// Refine set: the candidates whose screened loss is within kRefineBand of the minimum, lowest loss first (equal
+// losses: lower index first).  A set of one needs no second look.  A set larger than min(kMaxRefine, K/2) is not
+// evaluated either: the screened result stands as a whole, so that losses[] never mixes first and second
+// evaluations of candidates that close (the data is then flat to within the screening arithmetic: all scales
+// equal, for instance).  Each member gets the delta-weight slot of a candidate outside the set for the low part of
+// its split delta weights.
+__device__ void refine_select(const double* losses, int K, WorkspaceHeader* hdr) {      // one thread
+  hdr->refine_count = 0;
+  hdr->refine_done = 0;
+  if (hdr->status != TLQ_OK || K < 2) return;
+  const double lmin = __ldcg(losses + hdr->best_idx);
+  if (!(lmin > 0.0) || !isfinite(lmin)) return;
+  const double limit = lmin * (1.0 + kRefineBand);
+  const int cap = K / 2 < kMaxRefine ? K / 2 : kMaxRefine;
+  int cand[kMaxRefine];
+  int n = 0;
+  for (int j = 0; j < K; ++j) {
+    const double lj = __ldcg(losses + j);      // written by other CTAs of this launch: read past L1
+    if (!(lj <= limit)) continue;
+    if (n == cap) return;                       // too many to tell apart: keep the screened result
+    int pos = n;                                // insertion by (loss, index); j ascends, so equal losses keep their order
+    while (pos > 0 && __ldcg(losses + cand[pos - 1]) > lj) { cand[pos] = cand[pos - 1]; --pos; }
+    cand[pos] = j;
+    ++n;
+  }
+  if (n < 2) return;
+  int slot = 0;
+  for (int r = 0; r < n; ++r) {
+    bool used = true;
+    while (used) {            // next candidate index that is not in the set (K >= 2n: there is one)
+      used = false;
+      for (int q = 0; q < n; ++q) used = used || cand[q] == slot;
+      if (used) ++slot;
+    }
+    hdr->refine_cand[r] = cand[r];
+    hdr->refine_slot[r] = slot++;
+  }
+  hdr->refine_count = n;
+}
+
 // One CTA per candidate; the CTA that finishes last takes the argmin and copies the winning scale row.
 __global__ void __launch_bounds__(kRedThreads)
 loss_reduce_kernel(const float* __restrict__ partials, int64_t per_k, int K, const float* __restrict__ w_imp,
                    int64_t N, int64_t C2, const uint16_t* __restrict__ s_table, int64_t C1, WorkspaceHeader* hdr,
-                   double* __restrict__ losses, int32_t* __restrict__ best_idx, uint16_t* __restrict__ s_best) {
+                   double* __restrict__ losses, int32_t* __restrict__ best_idx, uint16_t* __restrict__ s_best,
+                   int pick_refine_set) {
   __shared__ double scratch[kRedThreads];
   __shared__ int best_sh;
   __shared__ int last_sh;
@@ -72,53 +113,13 @@ loss_reduce_kernel(const float* __restrict__ partials, int64_t per_k, int K, con
     hdr->best_idx = best;
     hdr->denom = denom;
     *best_idx = best;
+    if (pick_refine_set) refine_select(losses, K, hdr);
   }
   __syncthreads();
   if (s_best != nullptr) {
     const uint16_t* row = s_table + (int64_t)best_sh * C1;
     for (int64_t c = t; c < C1; c += kRedThreads) s_best[c] = row[c];
   }
-}
-
-// Refine set: the candidates whose screened loss is within kRefineBand of the minimum, lowest loss first (equal
-// losses: lower index first).  A set of one needs no second look.  A set larger than min(kMaxRefine, K/2) is not
-// evaluated either: the screened result stands as a whole, so that losses[] never mixes first and second
-// evaluations of candidates that close (the data is then flat to within the screening arithmetic: all scales
-// equal, for instance).  Each member gets the delta-weight slot of a candidate outside the set for the low part of
-// its split delta weights.
-__global__ void refine_select_kernel(const double* __restrict__ losses, int K, WorkspaceHeader* hdr) {
-  if (threadIdx.x != 0 || blockIdx.x != 0) return;
-  hdr->refine_count = 0;
-  hdr->refine_done = 0;
-  if (hdr->status != TLQ_OK || K < 2) return;
-  const double lmin = losses[hdr->best_idx];
-  if (!(lmin > 0.0) || !isfinite(lmin)) return;
-  const double limit = lmin * (1.0 + kRefineBand);
-  const int cap = K / 2 < kMaxRefine ? K / 2 : kMaxRefine;
-  int cand[kMaxRefine];
-  int n = 0;
-  for (int j = 0; j < K; ++j) {
-    const double lj = losses[j];
-    if (!(lj <= limit)) continue;
-    if (n == cap) return;                       // too many to tell apart: keep the screened result
-    int pos = n;                                // insertion by (loss, index); j ascends, so equal losses keep their order
-    while (pos > 0 && losses[cand[pos - 1]] > lj) { cand[pos] = cand[pos - 1]; --pos; }
-    cand[pos] = j;
-    ++n;
-  }
-  if (n < 2) return;
-  int slot = 0;
-  for (int r = 0; r < n; ++r) {
-    bool used = true;
-    while (used) {            // next candidate index that is not in the set (K >= 2n: there is one)
-      used = false;
-      for (int q = 0; q < n; ++q) used = used || cand[q] == slot;
-      if (used) ++slot;
-    }
-    hdr->refine_cand[r] = cand[r];
-    hdr->refine_slot[r] = slot++;
-  }
-  hdr->refine_count = n;
 }
 
 // One CTA per refined candidate: fixed-order fp64 sum of its partials; the CTA that finishes last takes the argmin
@@ -180,14 +181,9 @@ __global__ void per_token_reduce_kernel(const float* __restrict__ ptab, int K, i
 
 int launch_loss_reduce(const float* partials, int64_t per_k, int K, const float* w_imp, int64_t N, int64_t C2,
                        const uint16_t* s_table, int64_t C1, WorkspaceHeader* hdr, double* losses, int32_t* best_idx,
-                       uint16_t* s_best, cudaStream_t st) {
+                       uint16_t* s_best, bool pick_refine_set, cudaStream_t st) {
   loss_reduce_kernel<<<(unsigned)K, kRedThreads, 0, st>>>(partials, per_k, K, w_imp, N, C2, s_table, C1, hdr, losses, best_idx,
-                                               s_best);
-  return after_launch();
-}
-
-int launch_refine_select(const double* losses, int K, WorkspaceHeader* hdr, cudaStream_t st) {
-  refine_select_kernel<<<1, 32, 0, st>>>(losses, K, hdr);
+                                               s_best, pick_refine_set ? 1 : 0);
   return after_launch();
 }
 
