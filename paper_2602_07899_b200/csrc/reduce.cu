@@ -27,22 +27,22 @@ __device__ __forceinline__ double block_sum_fixed(double v, double* scratch) {
 // evaluations of candidates that close (the data is then flat to within the screening arithmetic: all scales
 // equal, for instance).  Each member gets the delta-weight slot of a candidate outside the set for the low part of
 // its split delta weights.
-__device__ void refine_select(const double* losses, int K, WorkspaceHeader* hdr) {      // one thread
+__device__ void refine_select(const double* losses /* a shared-memory copy */, int K, WorkspaceHeader* hdr) {  // one thread
   hdr->refine_count = 0;
   hdr->refine_done = 0;
   if (hdr->status != TLQ_OK || K < 2) return;
-  const double lmin = __ldcg(losses + hdr->best_idx);
+  const double lmin = losses[hdr->best_idx];
   if (!(lmin > 0.0) || !isfinite(lmin)) return;
   const double limit = lmin * (1.0 + kRefineBand);
   const int cap = K / 2 < kMaxRefine ? K / 2 : kMaxRefine;
   int cand[kMaxRefine];
   int n = 0;
   for (int j = 0; j < K; ++j) {
-    const double lj = __ldcg(losses + j);      // written by other CTAs of this launch: read past L1
+    const double lj = losses[j];
     if (!(lj <= limit)) continue;
     if (n == cap) return;                       // too many to tell apart: keep the screened result
     int pos = n;                                // insertion by (loss, index); j ascends, so equal losses keep their order
-    while (pos > 0 && __ldcg(losses + cand[pos - 1]) > lj) { cand[pos] = cand[pos - 1]; --pos; }
+    while (pos > 0 && losses[cand[pos - 1]] > lj) { cand[pos] = cand[pos - 1]; --pos; }
     cand[pos] = j;
     ++n;
   }
@@ -97,12 +97,14 @@ loss_reduce_kernel(const float* __restrict__ partials, int64_t per_k, int K, con
   __syncthreads();
   if (last_sh == 0) return;
 
+  __threadfence();
+  if (t < K) scratch[t] = __ldcg(losses + t);      // written by other CTAs: read past L1 (K <= TLQ_MAX_GRID)
+  __syncthreads();
   if (t == 0) {
-    __threadfence();
     int best = -1;
     double bv = __longlong_as_double(0x7FF0000000000000LL);
     for (int j = 0; j < K; ++j) {
-      const double lj = __ldcg(losses + j);      // written by other CTAs: read past L1
+      const double lj = scratch[j];
       if (lj < bv) { bv = lj; best = j; }
     }
     if (best < 0) {
@@ -113,7 +115,7 @@ loss_reduce_kernel(const float* __restrict__ partials, int64_t per_k, int K, con
     hdr->best_idx = best;
     hdr->denom = denom;
     *best_idx = best;
-    if (pick_refine_set) refine_select(losses, K, hdr);
+    if (pick_refine_set) refine_select(scratch, K, hdr);
   }
   __syncthreads();
   if (s_best != nullptr) {
