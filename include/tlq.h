@@ -90,8 +90,8 @@ extern "C" {
                                                faster inside a benchmark step). */
 
 #define TLQ_FLAG_NO_REFINE 8u                /* tlq_scale_search_layer, group mode: skip the refine pass.  By default,
-                                               when other candidates' losses come within 1e-4 (relative) of the
-                                               smallest, those candidates (if there are no more than four, and no
+                                               when other candidates' losses come within 1e-4 (relative; wider
+                                               below 1024 output channels: 3.2e-3 / sqrt(C2)) of the smallest, those candidates (if there are no more than four, and no
                                                more than K/2, of them: a flatter loss curve keeps its first result)
                                                are evaluated a second time with delta weights split into two bf16
                                                parts and short tensor-core accumulation chunks summed in registers

@@ -386,7 +386,7 @@ static int search_impl(const void* X, const void* X_ref, int64_t N, int64_t C1, 
   const bool refine =
       cfg->mode == TLQ_W4A16_ASYM_GROUP && !two_stream && K >= 2 && (cfg->flags & TLQ_FLAG_NO_REFINE) == 0;
   if ((rc = launch_loss_reduce(L.partials, used.partials_per_k, K, w_imp, N, C2, L.s, C1, L.hdr, losses, best_idx,
-                               reinterpret_cast<uint16_t*>(s_best), refine, st)) != TLQ_OK)
+                               reinterpret_cast<uint16_t*>(s_best), refine ? refine_band(C2) : 0.0, st)) != TLQ_OK)
     return rc;
   // Candidates too close to the minimum for the screening arithmetic to order are evaluated again, more exactly; the
   // set is chosen on the device, so the kernels are enqueued regardless and return at once when it is empty.

@@ -3,6 +3,7 @@
 
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
+#include <math.h>
 #include <stdint.h>
 
 #include "tlq.h"
@@ -234,17 +235,23 @@ int launch_top_mask(const float* imp, int64_t N, int64_t k_sel, uint8_t* mask, c
 // reduce.cu
 int launch_loss_reduce(const float* partials, int64_t per_k, int K, const float* w_imp, int64_t N, int64_t C2,
                        const uint16_t* s_table, int64_t C1, WorkspaceHeader* hdr, double* losses, int32_t* best_idx,
-                       uint16_t* s_best, bool pick_refine_set /* also fill hdr's refine set: 2 .. min(kMaxRefine, K/2)
-                       candidates, or none */, cudaStream_t st);
+                       uint16_t* s_best, double refine_band /* > 0: also fill hdr's refine set with the candidates
+                       within this relative distance of the minimum: 2 .. min(kMaxRefine, K/2) of them, or none */,
+                       cudaStream_t st);
 int launch_per_token_reduce(const float* ptab /*[K,otiles,Npad]*/, int K, int64_t otiles, int64_t Npad, int64_t N,
                             float* per_token /*[K,N]*/, cudaStream_t st);
 
 // Refine pass of the group-mode search (16-bit activations).  The screening GEMM sees delta weights rounded to bf16
-// and accumulates each output over all of C1 in the tensor core's fp32 accumulator, which shifts a loss by up to
-// 6e-5 relative; when two candidates are closer than that, the candidates within kRefineBand of the minimum are
-// evaluated again with split delta weights (bf16 high + bf16 low part) and short accumulation chunks summed outside
-// the tensor core, and the argmin is taken on those values.
-constexpr double kRefineBand = 1.0e-4;
+// and accumulates each output over all of C1 in the tensor core's fp32 accumulator.  The accumulation pulls a loss
+// down by up to 6e-5 relative (C1 up to 29568).  The rounding of a delta weight is shared by every token, so it
+// averages out over the C2 output channels only: about 2 * 2^-9 / sqrt(3 * C2) of the loss when one input channel
+// dominates (2.3e-4 measured at C2 = 72, at most 6e-5 in total at C2 >= 256 on 7B/72B-class layers).  Candidates
+// closer to the minimum than refine_band(C2) are evaluated again with split delta weights (bf16 high + bf16 low
+// part) and short accumulation chunks summed outside the tensor core, and the argmin is taken on those values.
+inline double refine_band(int64_t C2) {
+  const double by_rows = 3.2e-3 / sqrt((double)C2);      // 1e-4 from 1024 output channels on, 2e-4 at 256
+  return by_rows > 1.0e-4 ? by_rows : 1.0e-4;
+}
 // reduce.cu: refined losses from the fp64 partials [kMaxRefine][per_r]; rewrites losses[k] of the refined
 // candidates, the argmin and the winning scale row
 int launch_refine_finish(const double* partials, int64_t per_r, const uint16_t* s_table, int64_t C1,

@@ -21,19 +21,20 @@ __device__ __forceinline__ double block_sum_fixed(double v, double* scratch) {
   return scratch[0];
 }
 
-// Refine set: the candidates whose screened loss is within kRefineBand of the minimum, lowest loss first (equal
+// Refine set: the candidates whose screened loss is within `band` (relative) of the minimum, lowest loss first (equal
 // losses: lower index first).  A set of one needs no second look.  A set larger than min(kMaxRefine, K/2) is not
 // evaluated either: the screened result stands as a whole, so that losses[] never mixes first and second
 // evaluations of candidates that close (the data is then flat to within the screening arithmetic: all scales
 // equal, for instance).  Each member gets the delta-weight slot of a candidate outside the set for the low part of
 // its split delta weights.
-__device__ void refine_select(const double* losses /* a shared-memory copy */, int K, WorkspaceHeader* hdr) {  // one thread
+__device__ void refine_select(const double* losses /* a shared-memory copy */, int K, double band,
+                              WorkspaceHeader* hdr) {      // one thread
   hdr->refine_count = 0;
   hdr->refine_done = 0;
   if (hdr->status != TLQ_OK || K < 2) return;
   const double lmin = losses[hdr->best_idx];
   if (!(lmin > 0.0) || !isfinite(lmin)) return;
-  const double limit = lmin * (1.0 + kRefineBand);
+  const double limit = lmin * (1.0 + band);
   const int cap = K / 2 < kMaxRefine ? K / 2 : kMaxRefine;
   int cand[kMaxRefine];
   int n = 0;
@@ -66,7 +67,7 @@ __global__ void __launch_bounds__(kRedThreads)
 loss_reduce_kernel(const float* __restrict__ partials, int64_t per_k, int K, const float* __restrict__ w_imp,
                    int64_t N, int64_t C2, const uint16_t* __restrict__ s_table, int64_t C1, WorkspaceHeader* hdr,
                    double* __restrict__ losses, int32_t* __restrict__ best_idx, uint16_t* __restrict__ s_best,
-                   int pick_refine_set) {
+                   double refine_band) {
   __shared__ double scratch[kRedThreads];
   __shared__ int best_sh;
   __shared__ int last_sh;
@@ -115,7 +116,7 @@ loss_reduce_kernel(const float* __restrict__ partials, int64_t per_k, int K, con
     hdr->best_idx = best;
     hdr->denom = denom;
     *best_idx = best;
-    if (pick_refine_set) refine_select(scratch, K, hdr);
+    if (refine_band > 0.0) refine_select(scratch, K, refine_band, hdr);
   }
   __syncthreads();
   if (s_best != nullptr) {
@@ -183,9 +184,9 @@ __global__ void per_token_reduce_kernel(const float* __restrict__ ptab, int K, i
 
 int launch_loss_reduce(const float* partials, int64_t per_k, int K, const float* w_imp, int64_t N, int64_t C2,
                        const uint16_t* s_table, int64_t C1, WorkspaceHeader* hdr, double* losses, int32_t* best_idx,
-                       uint16_t* s_best, bool pick_refine_set, cudaStream_t st) {
+                       uint16_t* s_best, double refine_band, cudaStream_t st) {
   loss_reduce_kernel<<<(unsigned)K, kRedThreads, 0, st>>>(partials, per_k, K, w_imp, N, C2, s_table, C1, hdr, losses, best_idx,
-                                               s_best, pick_refine_set ? 1 : 0);
+                                               s_best, refine_band);
   return after_launch();
 }
 

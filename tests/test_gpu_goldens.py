@@ -104,13 +104,15 @@ def test_full_size_search_matches_stored_oracle(tlq, layer_data, cell, lin_name)
     assert best == int(g["best"]), (best, int(g["best"]), float(g["gap"]))
     assert best == int(np.argmin(losses))
     assert np.array_equal(s_best, g["scale_best"])
-    if cfgw.mode == "w4a16" and float(g["gap"]) < 7e-5:
+    # the refine pass takes on candidates within this relative distance of the screened minimum
+    band = max(1e-4, 3.2e-3 / np.sqrt(lin.c_out))
+    if cfgw.mode == "w4a16" and float(g["gap"]) < band - 3e-5:
         # close enough for the second, more exact evaluation to have run on the two best candidates: their losses
         # must then match the oracle's to its accuracy, not just to the screening tolerance
         assert n_refined >= 2
         top2 = np.argsort(g["losses"], kind="stable")[:2]
         np.testing.assert_allclose(losses[top2], g["losses"][top2], rtol=REFINED_RTOL)
-    if cfgw.mode != "w4a16" or float(g["gap"]) > 2e-4:
+    if cfgw.mode != "w4a16" or float(g["gap"]) > band + 1e-4:
         assert n_refined == 0
 
 

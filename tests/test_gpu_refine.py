@@ -53,7 +53,12 @@ def search(tlq, xb, wb, w32, group, n_grid, flags=0):
 
 
 @pytest.mark.parametrize("n,c1,c2,group,n_grid,seed", [(384, 1024, 256, 128, 12, 301), (300, 4096, 200, 64, 8, 302),
-                                                       (1100, 8192, 384, 128, 6, 303)])
+                                                       (1100, 8192, 384, 128, 6, 303),
+                                                       # ragged everywhere: 17 k-blocks (chunks of 4, 4, 4, 4, 1), a
+                                                       # last output tile of 2 channels, K = 4 (two spare slots)
+                                                       (257, 1088, 130, 64, 4, 304),
+                                                       # one and a half k-blocks, one chunk
+                                                       (200, 96, 72, 32, 5, 306)])
 def test_near_ties_are_decided_like_the_oracle(tlq, n, c1, c2, group, n_grid, seed):
     xb, wb, imp = wl.small_case(seed, n, c1, c2, n_outlier=2)
     base = orc.scale_search(xb, wb, imp, "w4a16", group, n_grid)
@@ -75,6 +80,10 @@ def test_near_ties_are_decided_like_the_oracle(tlq, n, c1, c2, group, n_grid, se
         np.testing.assert_allclose(losses[[a, b]], losses_ref[[a, b]], rtol=REFINED_RTOL)
         np.testing.assert_allclose(losses, losses_ref, rtol=2e-3)
         assert np.array_equal(s_best, orc.f32_to_bf16_bits(ref["scales"][best]))
+        # the pass does not depend on which screening kernel ran before it
+        best_n, losses_n, n_n, _ = search(tlq, xb, wb, w32, group, n_grid, flags=tlq.FLAG_GEMM_NARROW_TILES)
+        assert best_n == best and n_n == n_refined
+        np.testing.assert_allclose(losses_n[[a, b]], losses_ref[[a, b]], rtol=REFINED_RTOL)
         # the same call without the pass: same losses to the screening tolerance, argmin not asserted
         best0, losses0, n0, _ = search(tlq, xb, wb, w32, group, n_grid, flags=tlq.FLAG_NO_REFINE)
         assert n0 == 0
