@@ -46,6 +46,7 @@ extern "C" {
 #define TLQ_ERR_CUDA (-6)        /* a CUDA runtime / driver call failed (no device, launch error) */
 #define TLQ_ERR_TIMEOUT (-7)     /* device: a bounded barrier wait expired; results are invalid */
 #define TLQ_ERR_NONFINITE (-8)   /* device: every candidate's loss was non-finite */
+#define TLQ_ERR_OVERRUN (-9)     /* device: a guard word between workspace regions changed (TLQ_FLAG_DEBUG_CANARIES) */
 
 /* tlq_config.mode */
 #define TLQ_W4A16_ASYM_GROUP 0 /* weights: w_bits (2..8) asymmetric, one step + integer zero-point per
@@ -102,6 +103,15 @@ extern "C" {
                                                candidate is that close, and about four screening-candidates' time per
                                                re-evaluated candidate when some are.  Not run by the two-stream call
                                                nor in the symmetric modes (whose integer accumulation is exact). */
+
+#define TLQ_FLAG_DEBUG_CANARIES 16u          /* tlq_scale_search_layer (both forms), tlq_apply_layer: a debugging aid.
+                                               Every region of the workspace is followed by 256 bytes of guard words,
+                                               written when the call starts and compared when it ends; a guard that
+                                               changed sets the status word to TLQ_ERR_OVERRUN (and the header's second
+                                               int32 to 100 + the index of the guard), which shows a kernel writing
+                                               past the end of its region.  The flag is part of the configuration, so
+                                               the *_workspace_bytes() calls account for the guards.  Two tiny extra
+                                               launches per call; results are unchanged. */
 
 #define TLQ_MAX_GRID 64
 
@@ -257,6 +267,21 @@ int tlq_read_status(const void* workspace, void* stream);
  * device context is as usable as before: no fault, no trap, no unbounded loop.
  */
 int tlq_selftest_bounded_wait(void* workspace, size_t workspace_bytes, int64_t limit_cycles, void* stream);
+
+/*
+ * Diagnostics for TLQ_FLAG_DEBUG_CANARIES (the paper has no counterpart).  kind: 0 = the workspace of
+ * tlq_scale_search_layer, 1 = of tlq_apply_layer; cfg must carry the flag.
+ * tlq_debug_canary_offsets (host only, no device is touched): writes the byte offset of each guard (256 bytes each)
+ * into offsets[0 .. max_offsets) (host; may be NULL) and returns how many guards the layout has, or a negative
+ * TLQ_ERR_*.
+ * tlq_debug_check_canaries: compares the guards of a workspace that a flagged call has left behind once more (for
+ * instance after other work that might have scribbled on it); the outcome goes to the status word like the call's own
+ * check.  It does not clear the status word first.
+ */
+int tlq_debug_canary_offsets(int kind, int64_t N, int64_t C1, int64_t C2, const tlq_config* cfg,
+                             uint64_t* offsets /* host */, int max_offsets);
+int tlq_debug_check_canaries(int kind, int64_t N, int64_t C1, int64_t C2, const tlq_config* cfg, void* workspace,
+                             size_t workspace_bytes, void* stream);
 
 /*
  * Diagnostic (the paper has no counterpart): what the library measured about the current device's L2.  The L2 of this

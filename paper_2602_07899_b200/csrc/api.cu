@@ -30,7 +30,7 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 int check_cfg(const tlq_config* cfg, int64_t C1, bool need_quantizer = true) {
   if (cfg == nullptr || cfg->struct_size != sizeof(tlq_config)) return TLQ_ERR_INVALID_ARG;
   if ((cfg->flags & ~(uint32_t)(TLQ_FLAG_SKIP_ZERO_WEIGHT_TOKENS | TLQ_FLAG_GEMM_CTA_PAIRS | TLQ_FLAG_GEMM_NARROW_TILES |
-                                 TLQ_FLAG_NO_REFINE)) != 0)
+                                 TLQ_FLAG_NO_REFINE | TLQ_FLAG_DEBUG_CANARIES)) != 0)
     return TLQ_ERR_INVALID_ARG;
   if (cfg->n_grid < 1 || cfg->n_grid > TLQ_MAX_GRID) return TLQ_ERR_SHAPE;
   if (cfg->stat_mode < TLQ_STAT_MEAN_ABS || cfg->stat_mode > TLQ_STAT_MASKED_MAX) return TLQ_ERR_INVALID_ARG;
@@ -60,15 +60,24 @@ int have_device() {
 }
 
 // Carves consecutive 256-byte aligned regions out of a workspace (or only measures when base is null).
+// With `guarded` every region is followed by kGuardBytes that no kernel may write (TLQ_FLAG_DEBUG_CANARIES): a
+// pattern is put there when a call starts and verified when it ends.
 struct Carver {
   uint8_t* base;
   size_t off;
-  explicit Carver(void* b) : base(reinterpret_cast<uint8_t*>(b)), off(0) {}
+  bool guarded;
+  GuardList guards;
+  Carver(void* b, bool with_guards) : base(reinterpret_cast<uint8_t*>(b)), off(0), guarded(with_guards) { guards.n = 0; }
   template <typename T>
   T* take(size_t count, size_t align = 256) {
     off = align_up(off, align);
     T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
     off += count * sizeof(T);
+    if (guarded && guards.n < kMaxGuards) {
+      off = align_up(off, 16);
+      guards.off[guards.n++] = off;
+      off += kGuardBytes;
+    }
     return p;
   }
 };
@@ -92,6 +101,7 @@ struct SearchLayout {
   uint16_t* Xc;          // [n_pad, C1] packed activations
   double* refine_partials; // group mode: [kMaxRefine][refine_per_r] weighted tile sums of the refine pass
   int64_t refine_per_r;
+  GuardList guards;      // TLQ_FLAG_DEBUG_CANARIES: where the guard words between the regions are
   size_t bytes;
   GemmPlan plan;         // the mode's own GEMM
   GemmPlan plan_resident; // the tile-resident kernel's (all candidates per tile): symmetric modes and the two-stream search
@@ -101,7 +111,7 @@ struct SearchLayout {
 SearchLayout carve_search(void* ws, int64_t N, int64_t C1, int64_t C2, const tlq_config* cfg) {
   SearchLayout L{};
   const int K = cfg->n_grid;
-  Carver c(ws);
+  Carver c(ws, (cfg->flags & TLQ_FLAG_DEBUG_CANARIES) != 0);
   const bool i8 = cfg->mode == TLQ_W8A8_SYM;
   L.plan_resident = plan_search_gemm_i8(N, C1, C2, K);
   L.plan = i8 ? L.plan_resident : plan_search_gemm(N, C1, C2, K);
@@ -129,6 +139,7 @@ SearchLayout carve_search(void* ws, int64_t N, int64_t C1, int64_t C2, const tlq
     L.wc = c.take<float>((size_t)L.plan.n_pad);
     L.Xc = c.take<uint16_t>((size_t)L.plan.n_pad * C1, 1024);
   }
+  L.guards = c.guards;
   L.bytes = align_up(c.off, 256);
   return L;
 }
@@ -183,11 +194,12 @@ const char* tlq_status_string(int status) {
     case TLQ_ERR_CUDA: return "CUDA error or no CUDA device";
     case TLQ_ERR_TIMEOUT: return "device-side wait timed out";
     case TLQ_ERR_NONFINITE: return "all candidate losses are non-finite";
+    case TLQ_ERR_OVERRUN: return "a guard word between workspace regions was overwritten";
     default: return "unknown status";
   }
 }
 
-int tlq_version(void) { return 1008; }   // 1.8: refine pass of the group-mode search (TLQ_FLAG_NO_REFINE)
+int tlq_version(void) { return 1009; }   // 1.9: refine pass (TLQ_FLAG_NO_REFINE), workspace guard words (TLQ_FLAG_DEBUG_CANARIES)
 
 int64_t tlq_kernel_launch_count(void) { return (int64_t)g_launch_count; }
 
@@ -333,6 +345,7 @@ static int search_impl(const void* X, const void* X_ref, int64_t N, int64_t C1, 
   const int K = cfg->n_grid;
 
   TLQ_CUDA_TRY(cudaMemsetAsync(L.hdr, 0, sizeof(WorkspaceHeader), st));
+  if (L.guards.n > 0 && (rc = launch_canary_fill(workspace, L.guards, st)) != TLQ_OK) return rc;
   if ((rc = timing_mark(0, st)) != TLQ_OK) return rc;
   if ((rc = launch_channel_stats(Xb, N, C1, mask, cfg->stat_mode, L.stat_partials, st)) != TLQ_OK) return rc;
   if ((rc = launch_scale_table(L.stat_partials, stats_row_chunks(N), N, C1, cfg->stat_mode, K, L.x_stat, L.s, L.rs,
@@ -405,6 +418,7 @@ static int search_impl(const void* X, const void* X_ref, int64_t N, int64_t C1, 
   if (per_token_err != nullptr)
     if ((rc = launch_per_token_reduce(L.ptab, K, used.otiles * (resident ? 2 : 1), used.n_pad, N, per_token_err, st)) != TLQ_OK)
       return rc;
+  if (L.guards.n > 0 && (rc = launch_canary_check(workspace, L.guards, L.hdr, st)) != TLQ_OK) return rc;
   return timing_mark(4, st);
 }
 
@@ -436,11 +450,12 @@ struct ApplyLayout {
   float* u;
   int8_t* Xq;
   float* t;
+  GuardList guards;
   size_t bytes;
 };
 ApplyLayout carve_apply(void* ws, int64_t N, int64_t C1, int64_t C2, const tlq_config* cfg) {
   ApplyLayout L{};
-  Carver c(ws);
+  Carver c(ws, (cfg->flags & TLQ_FLAG_DEBUG_CANARIES) != 0);
   L.hdr = c.take<WorkspaceHeader>(1);
   if (cfg->mode == TLQ_W4A16_ASYM_GROUP) {
     L.dW = c.take<uint16_t>((size_t)C2 * C1, 1024);
@@ -450,6 +465,7 @@ ApplyLayout carve_apply(void* ws, int64_t N, int64_t C1, int64_t C2, const tlq_c
     L.Xq = c.take<int8_t>((size_t)N * C1, 1024);
     L.t = c.take<float>((size_t)N);
   }
+  L.guards = c.guards;
   L.bytes = align_up(c.off, 256);
   return L;
 }
@@ -482,17 +498,65 @@ int tlq_apply_layer(const void* X, int64_t N, int64_t C1, const void* W, int64_t
   const uint16_t* sb = reinterpret_cast<const uint16_t*>(s);
   const uint16_t* bb = reinterpret_cast<const uint16_t*>(bias);
   TLQ_CUDA_TRY(cudaMemsetAsync(L.hdr, 0, sizeof(WorkspaceHeader), st));
+  if (L.guards.n > 0 && (rc = launch_canary_fill(workspace, L.guards, st)) != TLQ_OK) return rc;
   if (cfg->mode == TLQ_W4A16_ASYM_GROUP) {
     if ((rc = launch_fakequant_group(Wb, sb, nullptr, 1, C2, C1, cfg->group_size, cfg->w_bits, L.dW, codes, steps,
                                      zeros, st)) != TLQ_OK)
       return rc;
-    return launch_apply_gemm_bf16(Xb, Wb, L.dW, bb, N, C1, C2, reinterpret_cast<uint16_t*>(Yq), L.hdr, st);
+    rc = launch_apply_gemm_bf16(Xb, Wb, L.dW, bb, N, C1, C2, reinterpret_cast<uint16_t*>(Yq), L.hdr, st);
+  } else {
+    if ((rc = launch_fakequant_rows_i8(Wb, sb, 1, C2, C1, cfg->w_bits, L.Wq, L.u, st)) != TLQ_OK) return rc;
+    if ((rc = launch_actquant_i8(Xb, sb, nullptr, 1, N, C1, cfg->a_bits, L.Xq, L.t, nullptr, st)) != TLQ_OK) return rc;
+    if (codes != nullptr) TLQ_CUDA_TRY(cudaMemcpyAsync(codes, L.Wq, (size_t)C2 * C1, cudaMemcpyDeviceToDevice, st));
+    if (steps != nullptr)
+      TLQ_CUDA_TRY(cudaMemcpyAsync(steps, L.u, (size_t)C2 * sizeof(float), cudaMemcpyDeviceToDevice, st));
+    rc = launch_apply_gemm_i8(L.Xq, L.Wq, L.t, L.u, bb, N, C1, C2, reinterpret_cast<uint16_t*>(Yq), L.hdr, st);
   }
-  if ((rc = launch_fakequant_rows_i8(Wb, sb, 1, C2, C1, cfg->w_bits, L.Wq, L.u, st)) != TLQ_OK) return rc;
-  if ((rc = launch_actquant_i8(Xb, sb, nullptr, 1, N, C1, cfg->a_bits, L.Xq, L.t, nullptr, st)) != TLQ_OK) return rc;
-  if (codes != nullptr) TLQ_CUDA_TRY(cudaMemcpyAsync(codes, L.Wq, (size_t)C2 * C1, cudaMemcpyDeviceToDevice, st));
-  if (steps != nullptr) TLQ_CUDA_TRY(cudaMemcpyAsync(steps, L.u, (size_t)C2 * sizeof(float), cudaMemcpyDeviceToDevice, st));
-  return launch_apply_gemm_i8(L.Xq, L.Wq, L.t, L.u, bb, N, C1, C2, reinterpret_cast<uint16_t*>(Yq), L.hdr, st);
+  if (rc != TLQ_OK) return rc;
+  if (L.guards.n > 0) rc = launch_canary_check(workspace, L.guards, L.hdr, st);
+  return rc;
+}
+
+// The guard words of a workspace laid out for (kind, N, C1, C2, cfg): kind 0 = search, 1 = apply.
+static int guards_of(int kind, int64_t N, int64_t C1, int64_t C2, const tlq_config* cfg, void* ws, GuardList* out,
+                     size_t* bytes) {
+  if (kind != 0 && kind != 1) return TLQ_ERR_INVALID_ARG;
+  if (N < 1 || C2 < 1) return TLQ_ERR_SHAPE;
+  const int rc = check_cfg(cfg, C1);
+  if (rc != TLQ_OK) return rc;
+  if ((cfg->flags & TLQ_FLAG_DEBUG_CANARIES) == 0) return TLQ_ERR_INVALID_ARG;
+  if (kind == 0) {
+    const SearchLayout L = carve_search(ws, N, C1, C2, cfg);
+    *out = L.guards; *bytes = L.bytes;
+  } else {
+    const ApplyLayout L = carve_apply(ws, N, C1, C2, cfg);
+    *out = L.guards; *bytes = L.bytes;
+  }
+  return TLQ_OK;
+}
+
+int tlq_debug_canary_offsets(int kind, int64_t N, int64_t C1, int64_t C2, const tlq_config* cfg, uint64_t* offsets,
+                             int max_offsets) {
+  GuardList g;
+  size_t bytes = 0;
+  const int rc = guards_of(kind, N, C1, C2, cfg, nullptr, &g, &bytes);
+  if (rc != TLQ_OK) return rc;
+  for (int i = 0; i < g.n && i < max_offsets && offsets != nullptr; ++i) offsets[i] = g.off[i];
+  return g.n;
+}
+
+int tlq_debug_check_canaries(int kind, int64_t N, int64_t C1, int64_t C2, const tlq_config* cfg, void* workspace,
+                             size_t workspace_bytes, void* stream) {
+  if (workspace == nullptr) return TLQ_ERR_INVALID_ARG;
+  if (!aligned16(workspace)) return TLQ_ERR_ALIGN;
+  GuardList g;
+  size_t bytes = 0;
+  int rc = guards_of(kind, N, C1, C2, cfg, workspace, &g, &bytes);
+  if (rc != TLQ_OK) return rc;
+  if (workspace_bytes < bytes) return TLQ_ERR_WORKSPACE;
+  if ((rc = have_device()) != TLQ_OK) return rc;
+  return launch_canary_check(workspace, g, reinterpret_cast<WorkspaceHeader*>(workspace),
+                             reinterpret_cast<cudaStream_t>(stream));
 }
 
 int tlq_read_status(const void* workspace, void* stream) {

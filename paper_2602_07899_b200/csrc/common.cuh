@@ -267,6 +267,18 @@ int launch_search_gemm_refine(const uint16_t* X, const uint16_t* dW, const float
                               int64_t C2, int K, double* partials, WorkspaceHeader* hdr, const int32_t* n_live,
                               cudaStream_t st);
 
+// selftest.cu: guard words between the regions of a workspace (TLQ_FLAG_DEBUG_CANARIES).  fill writes a pattern that
+// depends on the guard's index and the word's position; check compares and, on the first difference it sees, sets
+// hdr->status = TLQ_ERR_OVERRUN and hdr->where = 100 + index of the guard (unless an earlier error is recorded).
+constexpr int kMaxGuards = 32;
+constexpr size_t kGuardBytes = 256;
+struct GuardList {
+  int n;
+  unsigned long long off[kMaxGuards];      // byte offset of each guard from the start of the workspace
+};
+int launch_canary_fill(void* workspace, const GuardList& guards, cudaStream_t st);
+int launch_canary_check(const void* workspace, const GuardList& guards, WorkspaceHeader* hdr, cudaStream_t st);
+
 // selftest.cu: one warp waits `limit_cycles` on a barrier nobody arrives on, then reports TLQ_ERR_TIMEOUT in `hdr`
 int launch_bounded_wait_selftest(WorkspaceHeader* hdr, long long limit_cycles, cudaStream_t st);
 

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_PKG, "libtlq.so")
 
 OK = 0
 ERR_INVALID_ARG, ERR_SHAPE, ERR_ALIGN, ERR_UNSUPPORTED = -1, -2, -3, -4
-ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_NONFINITE = -5, -6, -7, -8
+ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_NONFINITE, ERR_OVERRUN = -5, -6, -7, -8, -9
 W4A16_ASYM_GROUP, W8A8_SYM = 0, 1
 WA_SYM_CHANNEL = W8A8_SYM     # symmetric per-channel weights / per-token activations, w_bits and a_bits in 2..8
 STAT_MEAN_ABS, STAT_MAX_ABS, STAT_MASKED_MAX = 0, 1, 2
@@ -31,7 +31,8 @@ EXPORTS = (
     "tlq_status_string", "tlq_version", "tlq_token_importance", "tlq_scale_candidates_workspace_bytes",
     "tlq_scale_candidates", "tlq_scale_candidates_noalloc", "tlq_quantize_weights", "tlq_pack_codes4", "tlq_quantize_activations", "tlq_scale_search_workspace_bytes", "tlq_scale_search_layer", "tlq_scale_search_layer_two_stream",
     "tlq_apply_layer_workspace_bytes", "tlq_apply_layer", "tlq_read_status", "tlq_stage_timing_enable",
-    "tlq_stage_timing_drain", "tlq_kernel_launch_count", "tlq_selftest_bounded_wait", "tlq_debug_tile_walk", "tlq_debug_resident_walk", "tlq_l2_partition_info",
+    "tlq_stage_timing_drain", "tlq_kernel_launch_count", "tlq_selftest_bounded_wait", "tlq_debug_tile_walk", "tlq_debug_resident_walk", "tlq_l2_partition_info", "tlq_debug_canary_offsets",
+    "tlq_debug_check_canaries",
 )
 
 
@@ -51,6 +52,7 @@ FLAG_SKIP_ZERO_WEIGHT_TOKENS = 1
 FLAG_GEMM_CTA_PAIRS = 2
 FLAG_GEMM_NARROW_TILES = 4
 FLAG_NO_REFINE = 8
+FLAG_DEBUG_CANARIES = 16
 
 
 def config(mode: int = W4A16_ASYM_GROUP, w_bits: Optional[int] = None, a_bits: Optional[int] = None,
@@ -97,6 +99,10 @@ def _load() -> ctypes.CDLL:
     lib.tlq_selftest_bounded_wait.restype = i32
     lib.tlq_debug_tile_walk.argtypes = [i64, i64, i32, i32, i32, i32, i32, vp]
     lib.tlq_debug_tile_walk.restype = i32
+    lib.tlq_debug_canary_offsets.argtypes = [i32, i64, i64, i64, vp, vp, i32]
+    lib.tlq_debug_canary_offsets.restype = i32
+    lib.tlq_debug_check_canaries.argtypes = [i32, i64, i64, i64, vp, vp, sz, vp]
+    lib.tlq_debug_check_canaries.restype = i32
     lib.tlq_l2_partition_info.argtypes = [vp, vp]
     lib.tlq_l2_partition_info.restype = i32
     lib.tlq_debug_resident_walk.argtypes = [i64, i64, i32, i32, i32, vp]
@@ -299,6 +305,21 @@ def tlq_selftest_bounded_wait(workspace: torch.Tensor, limit_cycles: int = 2_000
     _check(lib.tlq_selftest_bounded_wait(_ptr(workspace), workspace.numel() * workspace.element_size(), int(limit_cycles), st),
            "tlq_selftest_bounded_wait")
     return int(lib.tlq_read_status(_ptr(workspace), st))
+
+
+def tlq_debug_canary_offsets(kind: int, N: int, C1: int, C2: int, cfg: Config):
+    """-> list of byte offsets of the guard words of a workspace laid out with FLAG_DEBUG_CANARIES (host only)."""
+    buf = (ctypes.c_uint64 * 32)()
+    n = int(lib.tlq_debug_canary_offsets(kind, N, C1, C2, ctypes.byref(cfg), buf, 32))
+    _check(min(n, 0), "tlq_debug_canary_offsets")
+    return [int(buf[i]) for i in range(n)]
+
+
+def tlq_debug_check_canaries(kind: int, N: int, C1: int, C2: int, cfg: Config, workspace: torch.Tensor,
+                             stream=None) -> None:
+    """Enqueue one more comparison of the guard words; read the outcome with tlq_read_status."""
+    _check(lib.tlq_debug_check_canaries(kind, N, C1, C2, ctypes.byref(cfg), _ptr(workspace), workspace.numel(),
+                                        _stream(stream)), "tlq_debug_check_canaries")
 
 
 def tlq_l2_partition_info():

@@ -31,7 +31,7 @@ def test_every_declared_symbol_is_exported(tlq):
     for n in names:
         assert hasattr(tlq.lib, n), n
     assert sorted(tlq.EXPORTS) == names
-    assert tlq.lib.tlq_version() == 1008
+    assert tlq.lib.tlq_version() == 1009
     assert tlq.status_string(0) == "ok" and "workspace" in tlq.status_string(tlq.ERR_WORKSPACE)
 
 
@@ -91,7 +91,7 @@ def test_host_validation_error_codes(tlq):
     assert L.tlq_scale_search_layer(a, 4, 128, a, 8, None, None, ctypes.byref(cm), a, 1 << 30, a, a, a, None,
                                     None) == tlq.ERR_INVALID_ARG
     # flags: unknown bits, token skipping without weights or with a per-token table, options the two-stream call rejects
-    assert L.tlq_scale_search_layer(a, 4, 128, a, 8, None, None, ctypes.byref(tlq.config(flags=16)), a, 1 << 30, a, a, a,
+    assert L.tlq_scale_search_layer(a, 4, 128, a, 8, None, None, ctypes.byref(tlq.config(flags=32)), a, 1 << 30, a, a, a,
                                     None, None) == tlq.ERR_INVALID_ARG
     skip = tlq.config(flags=tlq.FLAG_SKIP_ZERO_WEIGHT_TOKENS)
     assert L.tlq_scale_search_layer(a, 4, 128, a, 8, None, None, ctypes.byref(skip), a, 1 << 30, a, a, a, None,
@@ -164,3 +164,24 @@ def test_resident_kernel_work_items_cover_every_candidate_of_every_tile_once(tlq
             for blocked in (False, True):
                 v = tlq.tlq_debug_resident_walk(mtiles, otiles, K, min(grid, mtiles * otiles), blocked)
                 assert v.min() == 1 and v.max() == 1, (mtiles, otiles, K, grid, blocked)
+
+
+def test_guard_word_layout_is_consistent(tlq):
+    """Host only: the guards of a flagged layout are ascending, 16-byte aligned, 256 bytes apart at least, inside
+    the workspace size the flagged configuration reports; an unflagged configuration has none to report."""
+    for mode, kw in ((tlq.W4A16_ASYM_GROUP, dict(group_size=128)), (tlq.W8A8_SYM, {})):
+        for flags in (0, tlq.FLAG_SKIP_ZERO_WEIGHT_TOKENS):
+            plain = tlq.config(mode, flags=flags, **kw)
+            guarded = tlq.config(mode, flags=flags | tlq.FLAG_DEBUG_CANARIES, **kw)
+            for kind, size_of in ((0, tlq.lib.tlq_scale_search_workspace_bytes), (1, tlq.lib.tlq_apply_layer_workspace_bytes)):
+                n, c1, c2 = 1000, 512, 264
+                offs = tlq.tlq_debug_canary_offsets(kind, n, c1, c2, guarded)
+                total = int(size_of(n, c1, c2, ctypes.byref(guarded)))
+                assert len(offs) >= (8 if kind == 0 else 2)
+                assert all(o % 16 == 0 for o in offs)
+                assert all(b - a >= 256 for a, b in zip(offs, offs[1:]))
+                assert offs[0] >= 256 and offs[-1] + 256 <= total
+                assert total > int(size_of(n, c1, c2, ctypes.byref(plain)))      # some guards fit into alignment gaps
+                assert tlq.lib.tlq_debug_canary_offsets(kind, n, c1, c2, ctypes.byref(plain), None, 0) == tlq.ERR_INVALID_ARG
+    assert tlq.lib.tlq_debug_canary_offsets(2, 8, 128, 8, ctypes.byref(tlq.config(flags=tlq.FLAG_DEBUG_CANARIES)), None,
+                                            0) == tlq.ERR_INVALID_ARG
