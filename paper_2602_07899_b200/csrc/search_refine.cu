@@ -47,6 +47,7 @@ struct RefineArgs {
   int64_t N;
   int num_kb;              // ceil(C1 / 64)
   int64_t mtiles, otiles;
+  TileRaster raster;       // walk order inside one candidate (whole token range, or 2048-token blocks)
   const int32_t* n_live;   // device: live token count after compaction, or null (= N)
   const float* w_imp;      // [N] or null (uniform)
   double* partials;        // [kMaxRefine][otiles*mtiles*4]
@@ -107,8 +108,11 @@ gemm_refine_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
   const int64_t mt_live = (n_tokens + BM - 1) / BM;          // token tiles that hold tokens
   const int64_t tiles_per_r = args.otiles * mt_live;
   const int64_t num_tiles = (int64_t)n_refine * tiles_per_r;
-  // tile -> (entry of the refine set, output tile, token tile), token tiles fastest: the CTAs in flight share a
-  // few weight tiles and sweep the activations
+  // tile -> (entry of the refine set, then the screening kernels' walk inside the candidate: token tiles fastest
+  // while the activations fit in L2, blocks of 2048 tokens x 9 output tiles when they do not)
+  TileRaster raster = args.raster;
+  raster.mtiles = (int)mt_live;
+  if (raster.b == 1) raster.a = mt_live > 0 ? (int)mt_live : 1;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -119,7 +123,8 @@ gemm_refine_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
       for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         const int r = (int)(tile / tiles_per_r);
         const int64_t rem = tile - (int64_t)r * tiles_per_r;
-        const int ot = (int)(rem / mt_live), mt = (int)(rem % mt_live);
+        int mt, ot;
+        raster.decode(rem, mt, ot);
         const int k_hi = args.hdr->refine_cand[r], k_lo = args.hdr->refine_slot[r];
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!ptx::mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
@@ -197,7 +202,8 @@ gemm_refine_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
       const int r = (int)(tile / tiles_per_r);
       const int64_t rem = tile - (int64_t)r * tiles_per_r;
-      const int ot = (int)(rem / mt_live), mt = (int)(rem % mt_live);
+      int mt, ot;
+      raster.decode(rem, mt, ot);
       float sums[BN];
 #pragma unroll
       for (int j = 0; j < BN; ++j) sums[j] = 0.0f;
@@ -302,6 +308,7 @@ int launch_search_gemm_refine(const uint16_t* X, const uint16_t* dW, const float
   if (sms <= 0) return TLQ_ERR_CUDA;
   const int64_t max_tiles = (int64_t)kMaxRefine * a.mtiles * a.otiles;
   const unsigned grid = (unsigned)(max_tiles < sms ? max_tiles : sms);
+  a.raster = make_raster(a.mtiles, a.otiles, sms, N * C1 * 2, BM);
   gemm_refine_kernel<<<grid, kThreads, kSmemBytes, st>>>(tmA, tmB, a);
   return after_launch();
 }
