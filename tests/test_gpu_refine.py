@@ -96,6 +96,39 @@ def test_near_ties_are_decided_like_the_oracle(tlq, n, c1, c2, group, n_grid, se
     print(f"screening alone decided {screened_right} of {len(deltas)} near-ties like the oracle")
 
 
+def three_way_weights(per_token, base_w, d1, d2):
+    """float32 weights under which, with a, b, c the three best candidates by base_w, loss_b = loss_a * (1 + d1) and
+    loss_c = loss_a * (1 + d2): two linear conditions, two sign patterns to scale the tokens by."""
+    a, b, c = np.argsort(per_token @ base_w, kind="stable")[:3]
+    u1 = np.where(per_token[b] > per_token[a], -1.0, 1.0)
+    u2 = np.where(per_token[c] > per_token[a], -1.0, 1.0)
+    r1 = per_token[b] - (1 + d1) * per_token[a]
+    r2 = per_token[c] - (1 + d2) * per_token[a]
+    lhs = np.array([[np.dot(base_w * u1, r1), np.dot(base_w * u2, r1)], [np.dot(base_w * u1, r2), np.dot(base_w * u2, r2)]])
+    t = np.linalg.solve(lhs, -np.array([np.dot(base_w, r1), np.dot(base_w, r2)]))
+    assert np.abs(t).sum() < 0.9, t
+    return (base_w * (1.0 + t[0] * u1 + t[1] * u2)).astype(np.float32), [int(a), int(b), int(c)]
+
+
+@pytest.mark.parametrize("n,c1,c2,group,n_grid,seed", [(640, 2048, 256, 128, 10, 320), (384, 1024, 256, 128, 12, 322)])
+def test_three_candidates_near_tied(tlq, n, c1, c2, group, n_grid, seed):
+    """Three candidates within 1e-5: all three are evaluated again and come out in the oracle's order."""
+    xb, wb, imp = wl.small_case(seed, n, c1, c2, n_outlier=2)
+    base = orc.scale_search(xb, wb, imp, "w4a16", group, n_grid)
+    w32, abc = three_way_weights(np.asarray(base["per_token"], np.float64), np.asarray(imp, np.float64), 4e-6, -6e-6)
+    ref = orc.scale_search(xb, wb, w32, "w4a16", group, n_grid)
+    losses_ref = np.asarray(ref["losses"])
+    order = [int(i) for i in np.argsort(losses_ref, kind="stable")]
+    assert order[:3] == [abc[2], abc[0], abc[1]] and ref["best"] == abc[2]
+    gaps = (losses_ref[order[1:4]] - losses_ref[order[0]]) / losses_ref[order[0]]
+    assert abs(gaps[0] - 6e-6) < 3e-7 and abs(gaps[1] - 1e-5) < 3e-7 and gaps[2] > 1e-3
+    best, losses, n_refined, s_best = search(tlq, xb, wb, w32, group, n_grid)
+    assert n_refined == 3 and best == ref["best"]
+    assert [int(i) for i in np.argsort(losses, kind="stable")][:3] == order[:3]
+    np.testing.assert_allclose(losses[abc], losses_ref[abc], rtol=REFINED_RTOL)
+    assert np.array_equal(s_best, orc.f32_to_bf16_bits(ref["scales"][best]))
+
+
 def test_no_near_tie_means_no_second_evaluation(tlq):
     """Well separated candidates: the refine set stays empty and the results are those of the flagged call, bit for bit."""
     xb, wb, imp = wl.small_case(17, 515, 1088, 777, n_outlier=2)
